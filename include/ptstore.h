@@ -1,0 +1,231 @@
+/*
+ * ptstore.h — C ABI of the single-GPU prefix tensor store (sm_100a).
+ *
+ * The library keeps the K/V tensors of token prefixes as a trie of fixed-size token blocks
+ * ("incremental, tensor-level prefix storage": an object stores only what follows its longest
+ * common prefix with earlier objects — paper Section 4, first paragraph, and Section 4.1
+ * "Co-optimized compact metadata and fast prefix queries").  The trie is encoded as an
+ * open-addressing hash table of chained 64-bit block keys that lives in device memory.
+ *
+ * General conventions
+ *   - Every array argument is a DEVICE-ACCESSIBLE pointer (device memory, or pinned host memory that
+ *     is mapped into the device address space) unless the argument is marked "host".
+ *   - The library allocates no device memory (it does allocate a few hundred bytes of host memory
+ *     for the handle).  Pools and workspace are owned by the caller and must outlive the handle.
+ *   - Every call that takes a stream only ENQUEUES work on that stream and returns; results are
+ *     valid once the stream has reached that point.  Calls on one handle must be issued from one
+ *     host thread at a time and onto one stream (or streams the caller has ordered); the library
+ *     takes no lock.
+ *   - Return value: PTSTORE_OK (0) or a negative PTSTORE_E_* code for conditions the host can see
+ *     (bad arguments, CUDA launch errors).  Conditions only the device can see (pool exhausted,
+ *     table full, block-table entry out of range, refcount underflow) are OR-ed as PTSTORE_S_* bits
+ *     into a device status word; the kernel skips the offending access and carries on.  Nothing
+ *     traps, nothing prints.
+ *   - Layout ("RDMA-aware consolidation", Section 4.1: an increment is one contiguous region and each
+ *     tensor an (offset,size) segment of it):
+ *       chunk  = one block of one layer's K (or V): [block_tokens][num_kv_heads][head_dim] elements,
+ *                contiguous; chunk_bytes must be a multiple of 16.
+ *       block  = [num_layers][2 (K,V)][chunk], contiguous: block_bytes = 2*num_layers*chunk_bytes.
+ *       pool   = [n_blocks][block]; block ids 0..hbm_blocks-1 are the HBM tier, ids
+ *                hbm_blocks..hbm_blocks+host_blocks-1 are the host tier (id - hbm_blocks indexes
+ *                host_pool).
+ *       paged cache (vLLM style), per layer: K block b at layer_base[l] + b*block_stride_bytes,
+ *                V block b at layer_base[l] + kv_stride_bytes + b*block_stride_bytes.
+ */
+#ifndef PTSTORE_H
+#define PTSTORE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ptstore ptstore_t;      /* opaque */
+typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy default stream */
+
+/* host-visible return codes */
+#define PTSTORE_OK          0
+#define PTSTORE_E_INVAL    (-1)   /* null / misaligned pointer, size out of range, bad struct_size */
+#define PTSTORE_E_CUDA     (-2)   /* a CUDA runtime call or launch failed (see ptstore_last_cuda_error) */
+#define PTSTORE_E_NOMEM    (-3)   /* host allocation of the handle failed, or workspace too small */
+#define PTSTORE_E_LIMIT    (-4)   /* batch exceeds max_requests / max_batch_blocks given at create */
+
+/* bits of the device status word (ptstore_status) */
+#define PTSTORE_S_NOSPACE     0x1u   /* insert: HBM free ring ran dry, some blocks were denied */
+#define PTSTORE_S_TABLE_FULL  0x2u   /* insert/rebuild: no free slot found within table_slots probes */
+#define PTSTORE_S_BOUNDS      0x4u   /* a block id or block-table entry was out of range; access skipped */
+#define PTSTORE_S_STATE       0x8u   /* release would have driven a refcount below zero; skipped */
+
+/* flags of ptstore_lookup */
+#define PTSTORE_PIN       0x1u   /* refcount++ on every matched (request, block) pair */
+#define PTSTORE_NO_TOUCH  0x2u   /* do not refresh the LRU stamp of matched blocks */
+
+/* flags of ptstore_config_t */
+#define PTSTORE_COPY_VECTOR  0x0u  /* copy engine: 16-byte vector loads/stores (always used for the host tier) */
+#define PTSTORE_COPY_BULK    0x1u  /* copy engine: bulk-async copies through a shared-memory ring (HBM<->HBM) */
+
+/* tiers of ptstore_evict */
+#define PTSTORE_TIER_HBM   0
+#define PTSTORE_TIER_HOST  1
+
+typedef struct {
+  uint32_t struct_size;          /* sizeof(ptstore_config_t), checked */
+  uint32_t flags;                /* PTSTORE_COPY_* */
+  uint32_t num_layers, num_kv_heads, head_dim, elem_bytes;   /* bf16: elem_bytes = 2 */
+  uint32_t block_tokens;         /* tokens per block, >= 1 */
+  uint32_t max_requests;         /* largest R any call will pass */
+  uint64_t max_batch_blocks;     /* largest R*max_blocks any call will pass */
+  uint64_t salt;                 /* folded into the root key (model / namespace id) */
+  void*    hbm_pool;             /* device memory, hbm_blocks*block_bytes, 16-byte aligned */
+  void*    host_pool;            /* device-visible pointer of mapped pinned memory, or NULL */
+  uint32_t hbm_blocks;           /* >= 1 */
+  uint32_t host_blocks;          /* 0 = no host tier */
+  uint64_t table_slots;          /* hash-table slots (any integer > hbm_blocks+host_blocks) */
+  void*    workspace;            /* device memory, 256-byte aligned */
+  uint64_t workspace_bytes;      /* >= ptstore_workspace_bytes(cfg) */
+  int32_t  device;               /* CUDA device ordinal that owns pools and workspace */
+  int32_t  reserved;
+} ptstore_config_t;
+
+typedef struct {
+  void* const* layer_base;       /* DEVICE array [num_layers] of device pointers, each 16-byte aligned */
+  uint64_t kv_stride_bytes;      /* V plane offset inside a layer tensor; multiple of 16 */
+  uint64_t block_stride_bytes;   /* distance between consecutive blocks; >= chunk_bytes, multiple of 16 */
+  uint32_t num_blocks;           /* block-table entries must be in [0, num_blocks) */
+  uint32_t reserved;
+} ptstore_paged_cache_t;
+
+typedef struct {                 /* all counters are cumulative since create */
+  uint64_t epoch;                /* lookup + insert calls so far (the LRU clock) */
+  uint64_t live_nodes[2];        /* trie nodes per tier right now */
+  uint64_t free_blocks[2];       /* free-ring fill per tier right now */
+  uint64_t tombstones;           /* deleted slots not yet reclaimed by a rebuild */
+  uint64_t query_blocks;         /* full blocks presented to lookup */
+  uint64_t probes_issued;        /* keys actually searched by lookup */
+  uint64_t slots_visited;        /* table slots read by those searches */
+  uint64_t blocks_matched;       /* sum of matched lengths */
+  uint64_t blocks_fetched[2];    /* per source tier */
+  uint64_t blocks_inserted;
+  uint64_t blocks_denied;
+  uint64_t blocks_dropped[2];    /* deleted per tier */
+  uint64_t blocks_demoted;       /* HBM -> host */
+  uint64_t rebuilds;
+} ptstore_stats_t;
+
+/*
+ * Bytes of workspace ptstore_create needs for this configuration (table x2, per-block metadata,
+ * free rings, per-batch scratch).  Only the size fields of cfg are read.  Returns 0 if cfg is invalid.
+ * No paper counterpart: the paper couples its store to a pre-registered allocator (Section 5,
+ * second paragraph); here the caller pre-allocates instead.
+ */
+uint64_t ptstore_workspace_bytes(const ptstore_config_t* cfg /*host*/);
+
+/*
+ * Create an empty store (Section 4: an empty trie; free rings hold every block id in ascending
+ * order; LRU clock 0).  Enqueues the initialisation on `stream`.  *out receives a handle that
+ * ptstore_destroy frees.  Errors: E_INVAL (geometry, alignment, sizes), E_NOMEM, E_CUDA.
+ */
+int ptstore_create(const ptstore_config_t* cfg /*host*/, ptstore_t** out /*host*/, ptstore_stream_t stream);
+
+/* Free the handle.  Caller memory is not touched.  The caller syncs outstanding work first. */
+int ptstore_destroy(ptstore_t* st);
+
+/*
+ * Chained block keys (the "unique tensor IDs" an object inherits from its longest common prefix and
+ * then extends, Section 4.1): keys[r*max_blocks + i] for every full block i < min(full_blocks(r),
+ * max_blocks) of request r; other entries are written as 0.  A trailing partial block is ignored.
+ *   tokens  int32 [offsets[R]]   ragged token ids; request r is tokens[offsets[r] .. offsets[r+1])
+ *   offsets int64 [R+1]          non-decreasing, offsets[0] >= 0
+ * Auxiliary entry point for verification; lookup and insert hash internally.
+ */
+int ptstore_hash(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                 uint64_t* keys_out /*[R*max_blocks]*/, ptstore_stream_t stream);
+
+/*
+ * Batched longest-common-prefix query (Section 1 "one-shot LCP query"; Section 4.1: a store or load
+ * first finds the longest common prefix among all previously stored objects).
+ *   matched_blocks[r] = number of leading full blocks of request r present in the store, capped at
+ *                       max_blocks; matched tokens = matched_blocks[r] * block_tokens.
+ *   block_ids[r*max_blocks + j] = pool block id holding block j for j < matched_blocks[r], else -1.
+ * Advances the LRU clock by one; unless NO_TOUCH stamps every matched block; with PIN adds one
+ * reference per matched (request, block) pair (reused blocks are marked by a reference counter,
+ * Section 1).  Ids of pinned blocks stay valid until released; other ids only until the next
+ * insert or evict.
+ */
+int ptstore_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                   uint32_t flags, int32_t* matched_blocks /*[R]*/, int32_t* block_ids /*[R*max_blocks]*/,
+                   ptstore_stream_t stream);
+
+/*
+ * Load (Section 4.1: iterate over the ids of an object and bring each tensor to the GPU pointers
+ * the application supplies).  For every r, j < matched_blocks[r], layer l, s in {K,V}: copy one chunk
+ * from pool block block_ids[r*max_blocks+j] to block block_tables[r*max_blocks+j] of the paged cache.
+ * Host-tier blocks are read in place through the mapped pointer.  No metadata changes.
+ * Entries with an id or table entry out of range are skipped and raise S_BOUNDS.
+ */
+int ptstore_fetch(ptstore_t* st, const int32_t* block_ids, const int32_t* matched_blocks, int32_t R,
+                  int32_t max_blocks, const ptstore_paged_cache_t* dst /*host struct*/,
+                  const int32_t* block_tables /*[R*max_blocks]*/, ptstore_stream_t stream);
+
+/*
+ * Store (Section 4: a store saves only the increment after the longest common prefix; Section 4.1:
+ * the application supplies the GPU pointers of the new tensors).  Requests are taken as if one after
+ * the other in index order: a block whose prefix is already stored is reused (and stamped), otherwise
+ * a block id is popped from the front of the HBM free ring, the 2*num_layers chunks are copied from
+ * src block block_tables[r*max_blocks+j] into it and a trie node is created.  When the ring runs dry
+ * the remaining new blocks are denied (-1) and S_NOSPACE is raised; nothing is evicted implicitly.
+ *   block_ids  out [R*max_blocks]: id now holding block j (existing or new), -1 if denied / beyond length
+ *   new_blocks out [R]: nodes created on behalf of request r (the lowest request index that presents
+ *                       a new prefix creates it)
+ * Advances the LRU clock by one.
+ */
+int ptstore_insert(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                   const ptstore_paged_cache_t* src /*host struct*/, const int32_t* block_tables,
+                   int32_t* block_ids, int32_t* new_blocks, ptstore_stream_t stream);
+
+/*
+ * Drop one reference per (r, j < matched_blocks[r]) pair (the counterpart of PIN; Section 1: blocks
+ * of finished requests become evictable).  A count that is already zero stays zero and raises S_STATE.
+ */
+int ptstore_release(ptstore_t* st, const int32_t* block_ids, const int32_t* matched_blocks, int32_t R,
+                    int32_t max_blocks, ptstore_stream_t stream);
+
+/*
+ * Evict up to n_blocks least-recently-used unreferenced leaves of a tier (Section 1: LRU over blocks
+ * of finished requests; Section 4.1 "Access pattern-aware eviction policy": owned tensors are flushed
+ * to slower tiers).  Order: (LRU stamp ascending, deeper first, lower id first); a parent freed by the
+ * removal of its last child in the same call may follow it.
+ *   tier HOST, or tier HBM without a host pool: the node is deleted and its id appended to the back of
+ *     that tier's free ring.
+ *   tier HBM with a host pool: if the host ring holds fewer than n_blocks free ids, the shortfall is
+ *     first dropped from the host tier; then up to min(n_blocks, host free) HBM blocks are copied to
+ *     host blocks popped from the front of the host ring; the node keeps its place in the trie under
+ *     its new id and the HBM id goes to the back of the HBM ring.
+ *   n_evicted  out, device [2]: [0] = blocks taken out of `tier` (dropped or demoted), [1] = host-tier
+ *              blocks dropped beforehand to make room for a demotion (0 in the other cases)
+ *   victim_ids out, device [2*n_blocks] or NULL: former ids of the n_evicted[0] blocks in the order
+ *              taken, followed by the n_evicted[1] room-making drops in the order taken
+ */
+int ptstore_evict(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids,
+                  ptstore_stream_t stream);
+
+/* Synchronise `stream`, read the device status word into *status_out (host) and clear it. */
+int ptstore_status(ptstore_t* st, ptstore_stream_t stream, uint32_t* status_out /*host*/);
+
+/* Synchronise `stream` and copy the counters to *out (host). */
+int ptstore_stats(ptstore_t* st, ptstore_stream_t stream, ptstore_stats_t* out /*host*/);
+
+/* Number of this library's kernels launched through the handle so far (host counter, no sync). */
+uint64_t ptstore_launch_count(const ptstore_t* st);
+
+/* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
+int ptstore_last_cuda_error(const ptstore_t* st);
+
+/* Static text for a PTSTORE_E_* code. */
+const char* ptstore_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PTSTORE_H */

@@ -1,0 +1,435 @@
+// CPU oracle of the prefix tensor store — TEST INFRASTRUCTURE, not a product path.
+//
+// A plain, single-threaded restatement of what the prefix-hit path computes, used only by the tests,
+// the smoke check and the CPU-baseline leg of the benchmark.  It shares no code with the CUDA
+// library and never calls it.  Nodes are found by comparing TOKENS (a pointer trie whose children are
+// keyed by the token content of a block), never by hash, so that a key collision in the hashed GPU
+// table would show up as a disagreement rather than be reproduced.
+//
+// What it follows:
+//   - Incremental prefix storage: a store keeps only the blocks after the longest common prefix with
+//     anything stored before; prefixes form a trie (paper Section 4, summary paragraph; Section 1,
+//     contributions).
+//   - Flat metadata: an object is the id list of its longest common prefix plus its own new ids
+//     (Section 4.1, "Co-optimized compact metadata and fast prefix queries").
+//   - Load = iterate over the ids and copy each tensor to the pointers the application supplies
+//     (Section 4.1, same paragraph and "Fine-grain multi-level caching").
+//   - Reference counts on reused blocks and LRU eviction of blocks of finished requests (Section 1,
+//     third paragraph); owned tensors are flushed to slower tiers rather than dropped (Section 4.1,
+//     "Access pattern-aware eviction policy").
+// The paper fixes no hash function, allocator order or tie-break; those are readings, stated next to
+// the code that implements them.
+//
+// Pins (tests/test_oracle_*.py): longest-prefix result vs brute force over all stored sequences;
+// trie invariants; hash known answers, invertibility of mix and constants derived from sqrt/phi;
+// copies vs memcpy round trips with canaries; literal greedy eviction vs the sorted closed form;
+// allocation order closed form.  Parity unpinned: nothing exported here.
+
+#include <cstdint>
+#include <cstring>
+#include <deque>
+#include <map>
+#include <algorithm>
+#include <tuple>
+#include <vector>
+
+namespace {
+
+typedef uint64_t u64;
+
+// ---- chained block hash (reading: the paper names no hash; this one is fixed by the build) --------
+// Constants: C1 = floor(2^64/phi); C2 = frac(sqrt 2)*2^64 | 1; C3 = frac(sqrt 3)*2^64; C5 = frac(sqrt 5)*2^64.
+const u64 C1 = 0x9E3779B97F4A7C15ull;
+const u64 C2 = 0x6A09E667F3BCC909ull;
+const u64 C3 = 0xBB67AE8584CAA73Bull;
+const u64 C5 = 0x3C6EF372FE94F82Bull;
+
+u64 mix(u64 x) {
+  x ^= x >> 32;
+  x *= C3;
+  x ^= x >> 29;
+  x *= C5;
+  x ^= x >> 32;
+  return x;
+}
+// keys 0 and 1 are reserved (empty / deleted slot markers of the hashed table)
+u64 fix(u64 k) { return k < 2 ? k + 2 : k; }
+u64 root_key(u64 salt) { return fix(mix(salt ^ C2)); }
+u64 chain_key(u64 parent, u64 content) { return fix(mix(parent * C1 + content)); }
+// wrapping sum over the block of mix(token | position<<32, xor C1): order independent, position aware
+u64 content_hash(const int32_t* t, int B) {
+  u64 s = 0;
+  for (int j = 0; j < B; ++j) {
+    u64 w = (u64)(uint32_t)t[j] | ((u64)j << 32);
+    s += mix(w ^ C1);
+  }
+  return s;
+}
+
+enum { TIER_HBM = 0, TIER_HOST = 1 };
+enum { S_NOSPACE = 1, S_TABLE_FULL = 2, S_BOUNDS = 4, S_STATE = 8 };
+enum { F_PIN = 1, F_NO_TOUCH = 2 };
+
+struct Node {
+  Node* parent;
+  std::map<std::vector<int32_t>, Node*> children;   // keyed by the block's tokens
+  int32_t depth;       // block index inside its sequence (0 = first block)
+  int32_t block_id;    // pool block that holds its K/V
+  int tier;
+  int64_t refcount;
+  u64 last_use;
+  u64 key;             // chained key, computed for comparison with the GPU path only
+  u64 tag;             // tag mode: identity of the payload
+  std::vector<int32_t> tokens;
+};
+
+struct PagedCache {
+  uint8_t* const* layer_base;
+  u64 kv_stride, block_stride;
+  uint32_t num_blocks;
+};
+
+struct Oracle {
+  int layers, B;
+  u64 chunk_bytes, block_bytes, salt;
+  int32_t n[2];                       // blocks per tier
+  bool byte_mode;
+  std::vector<uint8_t> pool[2];
+  std::deque<int32_t> free_list[2];
+  std::vector<Node*> by_id;           // live node per block id, or null
+  std::map<u64, Node*> by_key;        // only to DETECT two token paths with one key
+  u64 collisions;
+  u64 epoch;
+  uint32_t status;
+  Node root;
+
+  uint8_t* block_ptr(int32_t id) {
+    if (id < n[0]) return pool[0].data() + (u64)id * block_bytes;
+    return pool[1].data() + (u64)(id - n[0]) * block_bytes;
+  }
+  int tier_of(int32_t id) const { return id < n[0] ? TIER_HBM : TIER_HOST; }
+  int full_blocks(const int64_t* off, int r, int maxB) const {
+    int64_t nb = (off[r + 1] - off[r]) / B;
+    return (int)std::min<int64_t>(nb, maxB);
+  }
+};
+
+void free_subtree(Node* nd) {
+  for (auto& kv : nd->children) { free_subtree(kv.second); delete kv.second; }
+  nd->children.clear();
+}
+
+// Key of the eviction order: smaller goes first (reading: LRU stamp, then deeper first, then lower id)
+typedef std::tuple<u64, int64_t, int32_t> EvKey;
+EvKey ev_key(const Node* nd) { return EvKey(nd->last_use, -(int64_t)nd->depth, nd->block_id); }
+
+void remove_node(Oracle* o, Node* nd) {           // delete a leaf, give its id back (back of the ring)
+  o->by_id[nd->block_id] = nullptr;
+  o->by_key.erase(nd->key);
+  o->free_list[nd->tier].push_back(nd->block_id);
+  nd->parent->children.erase(nd->tokens);
+  delete nd;
+}
+
+bool has_child_in_tier(const Node* nd, int tier) {
+  for (auto& kv : nd->children) if (kv.second->tier == tier) return true;
+  return false;
+}
+bool has_descendant_in_other_tier(const Node* nd, int tier) {
+  for (auto& kv : nd->children) {
+    if (kv.second->tier != tier) return true;
+    if (has_descendant_in_other_tier(kv.second, tier)) return true;
+  }
+  return false;
+}
+
+// ---- drop: literal greedy loop --------------------------------------------------------------------
+int drop_literal(Oracle* o, int tier, int n, int32_t* victims) {
+  int taken = 0;
+  while (taken < n) {
+    Node* best = nullptr;
+    for (Node* nd : o->by_id) {
+      if (!nd || nd->tier != tier || nd->refcount != 0 || !nd->children.empty()) continue;
+      if (!best || ev_key(nd) < ev_key(best)) best = nd;
+    }
+    if (!best) break;
+    if (victims) victims[taken] = best->block_id;
+    ++taken;
+    remove_node(o, best);
+  }
+  return taken;
+}
+// ---- drop: closed form (first n unreferenced nodes of the tier without a live descendant in the
+// other tier, in key order).  Equal to the greedy loop while refcount(parent) >= refcount(child) and
+// last_use(parent) >= last_use(child) hold; tests assert the equality on random tries.
+int drop_sorted(Oracle* o, int tier, int n, int32_t* victims) {
+  std::vector<Node*> cand;
+  for (Node* nd : o->by_id)
+    if (nd && nd->tier == tier && nd->refcount == 0 && !has_descendant_in_other_tier(nd, tier)) cand.push_back(nd);
+  std::sort(cand.begin(), cand.end(), [](Node* a, Node* b) { return ev_key(a) < ev_key(b); });
+  int taken = 0;
+  for (Node* nd : cand) {
+    if (taken >= n) break;
+    if (victims) victims[taken] = nd->block_id;
+    ++taken;
+    remove_node(o, nd);            // children sort before parents, so nd is a leaf by now
+  }
+  return taken;
+}
+
+void demote_node(Oracle* o, Node* nd) {           // HBM -> host, node stays in the trie
+  int32_t old_id = nd->block_id;
+  int32_t new_id = o->free_list[TIER_HOST].front();
+  o->free_list[TIER_HOST].pop_front();
+  if (o->byte_mode) std::memcpy(o->block_ptr(new_id), o->block_ptr(old_id), o->block_bytes);
+  o->by_id[old_id] = nullptr;
+  o->by_id[new_id] = nd;
+  nd->block_id = new_id;
+  nd->tier = TIER_HOST;
+  o->free_list[TIER_HBM].push_back(old_id);
+}
+int demote_literal(Oracle* o, int n, int32_t* victims) {
+  int taken = 0;
+  while (taken < n && !o->free_list[TIER_HOST].empty()) {
+    Node* best = nullptr;
+    for (Node* nd : o->by_id) {
+      if (!nd || nd->tier != TIER_HBM || nd->refcount != 0 || has_child_in_tier(nd, TIER_HBM)) continue;
+      if (!best || ev_key(nd) < ev_key(best)) best = nd;
+    }
+    if (!best) break;
+    if (victims) victims[taken] = best->block_id;
+    ++taken;
+    demote_node(o, best);
+  }
+  return taken;
+}
+int demote_sorted(Oracle* o, int n, int32_t* victims) {
+  std::vector<Node*> cand;
+  for (Node* nd : o->by_id)
+    if (nd && nd->tier == TIER_HBM && nd->refcount == 0) cand.push_back(nd);
+  std::sort(cand.begin(), cand.end(), [](Node* a, Node* b) { return ev_key(a) < ev_key(b); });
+  int taken = 0;
+  for (Node* nd : cand) {
+    if (taken >= n || o->free_list[TIER_HOST].empty()) break;
+    if (victims) victims[taken] = nd->block_id;
+    ++taken;
+    demote_node(o, nd);
+  }
+  return taken;
+}
+
+}  // namespace
+
+extern "C" {
+
+// exported pieces of the hash, for known-answer and property tests
+uint64_t oracle_mix(uint64_t x) { return mix(x); }
+uint64_t oracle_root(uint64_t salt) { return root_key(salt); }
+uint64_t oracle_chain(uint64_t p, uint64_t c) { return chain_key(p, c); }
+uint64_t oracle_content(const int32_t* t, int32_t B) { return content_hash(t, B); }
+
+void* oracle_create(int32_t layers, int32_t heads, int32_t dim, int32_t elem_bytes, int32_t block_tokens,
+                    uint64_t salt, int32_t hbm_blocks, int32_t host_blocks, int32_t byte_mode) {
+  Oracle* o = new Oracle();
+  o->layers = layers; o->B = block_tokens; o->salt = salt;
+  o->chunk_bytes = (u64)block_tokens * heads * dim * elem_bytes;
+  o->block_bytes = 2ull * layers * o->chunk_bytes;
+  o->n[0] = hbm_blocks; o->n[1] = host_blocks;
+  o->byte_mode = byte_mode != 0;
+  if (o->byte_mode) {
+    o->pool[0].assign((u64)hbm_blocks * o->block_bytes, 0);
+    o->pool[1].assign((u64)host_blocks * o->block_bytes, 0);
+  }
+  for (int32_t i = 0; i < hbm_blocks; ++i) o->free_list[0].push_back(i);                 // ascending ids
+  for (int32_t i = 0; i < host_blocks; ++i) o->free_list[1].push_back(hbm_blocks + i);
+  o->by_id.assign((size_t)hbm_blocks + host_blocks, nullptr);
+  o->collisions = 0; o->epoch = 0; o->status = 0;
+  o->root.parent = nullptr; o->root.depth = -1; o->root.block_id = -1; o->root.tier = -1;
+  o->root.refcount = 0; o->root.last_use = 0; o->root.key = root_key(salt); o->root.tag = 0;
+  return o;
+}
+
+void oracle_destroy(void* h) {
+  Oracle* o = (Oracle*)h;
+  free_subtree(&o->root);
+  delete o;
+}
+
+void oracle_hash(void* h, const int32_t* tokens, const int64_t* off, int32_t R, int32_t maxB, uint64_t* keys) {
+  Oracle* o = (Oracle*)h;
+  for (int r = 0; r < R; ++r) {
+    int nb = o->full_blocks(off, r, maxB);
+    u64 k = root_key(o->salt);
+    for (int j = 0; j < maxB; ++j) {
+      if (j < nb) { k = chain_key(k, content_hash(tokens + off[r] + (int64_t)j * o->B, o->B)); keys[(int64_t)r * maxB + j] = k; }
+      else keys[(int64_t)r * maxB + j] = 0;
+    }
+  }
+}
+
+// longest stored prefix of every request, block by block from the root
+void oracle_lookup(void* h, const int32_t* tokens, const int64_t* off, int32_t R, int32_t maxB, uint32_t flags,
+                   int32_t* matched, int32_t* ids) {
+  Oracle* o = (Oracle*)h;
+  o->epoch += 1;
+  for (int r = 0; r < R; ++r) {
+    int nb = o->full_blocks(off, r, maxB);
+    Node* cur = &o->root;
+    int m = 0;
+    for (; m < nb; ++m) {
+      const int32_t* t = tokens + off[r] + (int64_t)m * o->B;
+      auto it = cur->children.find(std::vector<int32_t>(t, t + o->B));
+      if (it == cur->children.end()) break;
+      cur = it->second;
+      ids[(int64_t)r * maxB + m] = cur->block_id;
+      if (!(flags & F_NO_TOUCH)) cur->last_use = o->epoch;
+      if (flags & F_PIN) cur->refcount += 1;
+    }
+    for (int j = m; j < maxB; ++j) ids[(int64_t)r * maxB + j] = -1;
+    matched[r] = m;
+  }
+}
+
+// byte copies pool -> paged cache
+void oracle_fetch(void* h, const int32_t* ids, const int32_t* matched, int32_t R, int32_t maxB,
+                  uint8_t* const* layer_base, uint64_t kv_stride, uint64_t block_stride, uint32_t num_blocks,
+                  const int32_t* bt) {
+  Oracle* o = (Oracle*)h;
+  int32_t total = o->n[0] + o->n[1];
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < matched[r] && j < maxB; ++j) {
+      int32_t id = ids[(int64_t)r * maxB + j], db = bt[(int64_t)r * maxB + j];
+      if (id < 0 || id >= total || db < 0 || (uint32_t)db >= num_blocks) { o->status |= S_BOUNDS; continue; }
+      const uint8_t* src = o->block_ptr(id);
+      for (int l = 0; l < o->layers; ++l)
+        for (int s = 0; s < 2; ++s)
+          std::memcpy(layer_base[l] + s * kv_stride + (u64)db * block_stride,
+                      src + ((u64)l * 2 + s) * o->chunk_bytes, o->chunk_bytes);
+    }
+}
+
+// sequential insert, request by request, block by block
+void oracle_insert(void* h, const int32_t* tokens, const int64_t* off, int32_t R, int32_t maxB,
+                   uint8_t* const* layer_base, uint64_t kv_stride, uint64_t block_stride, uint32_t num_blocks,
+                   const int32_t* bt, const uint64_t* tags, int32_t* ids, int32_t* new_blocks) {
+  Oracle* o = (Oracle*)h;
+  o->epoch += 1;
+  for (int r = 0; r < R; ++r) {
+    int nb = o->full_blocks(off, r, maxB);
+    for (int j = 0; j < maxB; ++j) ids[(int64_t)r * maxB + j] = -1;
+    new_blocks[r] = 0;
+    Node* cur = &o->root;
+    for (int j = 0; j < nb; ++j) {
+      const int32_t* t = tokens + off[r] + (int64_t)j * o->B;
+      std::vector<int32_t> blk(t, t + o->B);
+      auto it = cur->children.find(blk);
+      if (it != cur->children.end()) {
+        cur = it->second;
+        cur->last_use = o->epoch;
+        ids[(int64_t)r * maxB + j] = cur->block_id;
+        continue;
+      }
+      if (o->free_list[TIER_HBM].empty()) { o->status |= S_NOSPACE; break; }   // deny the rest of this request
+      int32_t sb = bt ? bt[(int64_t)r * maxB + j] : 0;
+      const bool copy = o->byte_mode && layer_base;              // no source cache given: metadata only
+      if (copy && (sb < 0 || (uint32_t)sb >= num_blocks)) { o->status |= S_BOUNDS; break; }
+      int32_t id = o->free_list[TIER_HBM].front();
+      o->free_list[TIER_HBM].pop_front();
+      Node* nd = new Node();
+      nd->parent = cur; nd->depth = j; nd->block_id = id; nd->tier = TIER_HBM; nd->refcount = 0;
+      nd->last_use = o->epoch; nd->key = chain_key(cur->key, content_hash(t, o->B));
+      nd->tag = tags ? tags[(int64_t)r * maxB + j] : 0;
+      nd->tokens = blk;
+      if (o->by_key.count(nd->key)) o->collisions += 1; else o->by_key[nd->key] = nd;
+      cur->children[blk] = nd;
+      o->by_id[id] = nd;
+      if (copy) {
+        uint8_t* dst = o->block_ptr(id);
+        for (int l = 0; l < o->layers; ++l)
+          for (int s = 0; s < 2; ++s)
+            std::memcpy(dst + ((u64)l * 2 + s) * o->chunk_bytes,
+                        layer_base[l] + s * kv_stride + (u64)sb * block_stride, o->chunk_bytes);
+      }
+      ids[(int64_t)r * maxB + j] = id;
+      new_blocks[r] += 1;
+      cur = nd;
+    }
+  }
+}
+
+void oracle_release(void* h, const int32_t* ids, const int32_t* matched, int32_t R, int32_t maxB) {
+  Oracle* o = (Oracle*)h;
+  int32_t total = o->n[0] + o->n[1];
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < matched[r] && j < maxB; ++j) {
+      int32_t id = ids[(int64_t)r * maxB + j];
+      if (id < 0 || id >= total || !o->by_id[id]) { o->status |= S_BOUNDS; continue; }
+      if (o->by_id[id]->refcount <= 0) { o->status |= S_STATE; continue; }
+      o->by_id[id]->refcount -= 1;
+    }
+}
+
+// mode 0: literal greedy loops; mode 1: sorted closed forms.
+// n_evicted[0] = blocks taken out of `tier` (dropped, or demoted to host); n_evicted[1] = host-tier
+// blocks dropped beforehand to make room for a demotion.  victims (2*n entries): the former ids of
+// the n_evicted[0] blocks in the order taken, followed by the n_evicted[1] room-making drops.
+void oracle_evict(void* h, int32_t tier, int32_t n, int32_t mode, int32_t* n_evicted, int32_t* victims) {
+  Oracle* o = (Oracle*)h;
+  if (n < 0) n = 0;
+  n_evicted[0] = n_evicted[1] = 0;
+  if (tier == TIER_HOST || o->n[1] == 0) {
+    n_evicted[0] = mode ? drop_sorted(o, tier, n, victims) : drop_literal(o, tier, n, victims);
+    return;
+  }
+  int host_free = (int)o->free_list[TIER_HOST].size();
+  int k = std::max(0, n - host_free);
+  std::vector<int32_t> dropped(k > 0 ? k : 1);
+  int nd = 0;
+  if (k > 0) nd = mode ? drop_sorted(o, TIER_HOST, k, dropped.data()) : drop_literal(o, TIER_HOST, k, dropped.data());
+  host_free = (int)o->free_list[TIER_HOST].size();
+  int want = std::min(n, host_free);
+  int taken = mode ? demote_sorted(o, want, victims) : demote_literal(o, want, victims);
+  if (victims) for (int i = 0; i < nd; ++i) victims[taken + i] = dropped[i];
+  n_evicted[0] = taken;
+  n_evicted[1] = nd;
+}
+
+uint32_t oracle_status(void* h) { Oracle* o = (Oracle*)h; uint32_t s = o->status; o->status = 0; return s; }
+uint64_t oracle_epoch(void* h) { return ((Oracle*)h)->epoch; }
+uint64_t oracle_collisions(void* h) { return ((Oracle*)h)->collisions; }
+int32_t oracle_free_count(void* h, int32_t tier) { return (int32_t)((Oracle*)h)->free_list[tier].size(); }
+void oracle_free_list(void* h, int32_t tier, int32_t* out) {
+  Oracle* o = (Oracle*)h; int i = 0;
+  for (int32_t id : o->free_list[tier]) out[i++] = id;
+}
+int32_t oracle_live_count(void* h, int32_t tier) {
+  Oracle* o = (Oracle*)h; int c = 0;
+  for (Node* nd : o->by_id) if (nd && nd->tier == tier) ++c;
+  return c;
+}
+// info[0..7] = live, refcount, last_use, depth, parent block id (-1 = root), key, tag, number of children
+void oracle_block_info(void* h, int32_t id, uint64_t* info) {
+  Oracle* o = (Oracle*)h;
+  Node* nd = (id >= 0 && id < (int32_t)o->by_id.size()) ? o->by_id[id] : nullptr;
+  if (!nd) { for (int i = 0; i < 8; ++i) info[i] = 0; return; }
+  info[0] = 1; info[1] = (u64)nd->refcount; info[2] = nd->last_use; info[3] = (u64)nd->depth;
+  info[4] = (u64)(int64_t)(nd->parent == &o->root ? -1 : nd->parent->block_id);
+  info[5] = nd->key; info[6] = nd->tag; info[7] = nd->children.size();
+}
+void oracle_block_tags(void* h, const int32_t* ids, int64_t n, uint64_t* out) {
+  Oracle* o = (Oracle*)h;
+  for (int64_t i = 0; i < n; ++i) {
+    int32_t id = ids[i];
+    Node* nd = (id >= 0 && id < (int32_t)o->by_id.size()) ? o->by_id[id] : nullptr;
+    out[i] = nd ? nd->tag : 0;
+  }
+}
+uint8_t* oracle_pool_ptr(void* h, int32_t tier) { Oracle* o = (Oracle*)h; return o->byte_mode ? o->pool[tier].data() : nullptr; }
+uint64_t oracle_block_bytes(void* h) { return ((Oracle*)h)->block_bytes; }
+// set a node's fields directly: lets property tests build arbitrary (still consistent) states
+void oracle_poke(void* h, int32_t id, int64_t refcount, uint64_t last_use) {
+  Oracle* o = (Oracle*)h;
+  if (id >= 0 && id < (int32_t)o->by_id.size() && o->by_id[id]) { o->by_id[id]->refcount = refcount; o->by_id[id]->last_use = last_use; }
+}
+
+}  // extern "C"
