@@ -1,0 +1,408 @@
+"""Benchmark of the prefix-hit path on B200.
+
+A step is one pass of the whole path over one batch of synthetic prompts:
+    lookup(PIN) -> fetch -> evict(what the batch will need) -> insert -> release
+on the Llama-3-8B KV shape (32 layers x 8 KV heads x 128, bf16, 16-token blocks), a 20,000-block store
+pool in HBM, 500 documents of 2k-6k tokens with Zipf(1.1) popularity, 64 prompts per batch, each a
+document plus a unique 64-256-token question.
+
+Prints ONE JSON line.  `value` is KV bytes moved by fetch and insert (read + write) divided by the
+time of the whole steps, inputs resident in HBM.  `e2e` repeats the measurement with the step's token
+ids / offsets / block tables copied from pinned host memory and its results copied back inside the
+timed region.  `roofline` is the fetch copy kernel alone against the measured HBM copy bandwidth.
+`cpu_baseline` is the CPU oracle timed on this machine on a bounded sample of the same stream.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--engine vector|bulk] ...
+Under torchrun (N > 1) every rank runs an independent replica on its own GPU (the path has no
+exchange step); rank 0 prints the aggregate.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_22648_b200 import workloads as W  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index, period=0.01):
+        self.index, self.period, self.rows, self.stop_flag, self.t = index, period, [], False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+        except Exception:
+            self.nv = None
+
+    def start(self):
+        if self.nv is None:
+            return
+        self.stop_flag = False
+        self.rows = []
+        self.t = threading.Thread(target=self._poll, daemon=True)
+        self.t.start()
+
+    def _poll(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                clk = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    rs = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    rs = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.rows.append((clk, rs))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        if self.nv is None or self.t is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"], "samples": 0}
+        self.stop_flag = True
+        self.t.join(timeout=2)
+        nv = self.nv
+        try:
+            mx = float(nv.nvmlDeviceGetMaxClockInfo(self.h, nv.NVML_CLOCK_SM))
+        except Exception:
+            mx = None
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4,
+                "hw_power_brake": 0x80}
+        reasons = set()
+        for _, rs in self.rows:
+            for name, bit in bits.items():
+                if rs & bit:
+                    reasons.add(name)
+        clk = [c for c, _ in self.rows]
+        return {"sm_mhz": float(np.median(clk)) if clk else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(clk)}
+
+
+# ---------------------------------------------------------------------------------------------------------
+class Llama8BServing:
+    """configs[1]: the workload the metric is quoted on."""
+    name = "llama3_8b_kv_pool20k_zipf1.1_batch64"
+
+    def __init__(self, args, rank):
+        import torch
+        from paper_2607_22648_b200 import binding as G
+        self.torch, self.G = torch, G
+        self.sh = W.LLAMA3_8B
+        self.batch, self.pool_blocks = args.batch, args.pool_blocks
+        self.stream = W.llama8b_stream(seed=W.BASE_SEED + 1 + 1000 * rank, n_docs=args.docs)
+        self.mb = self.stream.max_blocks
+        flags = (G.COPY_BULK if args.engine == "bulk" else G.COPY_VECTOR) | G.copy_variant(args.variant) | \
+            G.copy_ctas_per_sm(args.ctas_per_sm)
+        self.store = G.PTStore(self.sh.layers, self.sh.heads, self.sh.dim, self.sh.block_tokens, self.pool_blocks,
+                               max_requests=self.batch, max_batch_blocks=self.batch * self.mb, flags=flags)
+        self.rng = np.random.default_rng(W.BASE_SEED + 77 + rank)
+        self.steps = []
+        self.cache = None
+
+    def prepare(self, n_steps):
+        """Generate every batch up front (host + device copies) and size the paged cache for the largest."""
+        torch = self.torch
+        B = self.sh.block_tokens
+        raw, need_max = [], 0
+        for _ in range(n_steps):
+            seqs, _tags = self.stream.batch(self.batch)
+            need = sum(len(s) // B for s in seqs)
+            need_max = max(need_max, need)
+            raw.append((seqs, need))
+        self.cache_blocks = need_max + 16
+        self.cache = self.G.PagedKV(self.sh.layers, self.cache_blocks, self.sh.chunk_bytes)
+        words = self.sh.chunk_bytes // 4
+        for t in self.cache.tensors:                       # any bytes will do for timing; make them non-trivial
+            t.view(torch.int32).copy_(torch.randint(-2**31, 2**31 - 1, (2 * self.cache_blocks * words,), dtype=torch.int32,
+                                                    device="cuda").view(2, self.cache_blocks, words))
+        for seqs, need in raw:
+            toks, offs = W.ragged(seqs)
+            bt = W.shuffled_block_tables(self.rng, seqs, B, self.mb, self.cache_blocks)
+            nblk = np.array([len(s) // B for s in seqs], dtype=np.int64)
+            host = dict(tokens=torch.from_numpy(toks).pin_memory(), offsets=torch.from_numpy(offs).pin_memory(),
+                        bt=torch.from_numpy(bt).pin_memory())
+            devc = {k: v.cuda() for k, v in host.items()}
+            self.steps.append(dict(host=host, dev=devc, nblk=nblk, total_blocks=int(nblk.sum())))
+        R = self.batch
+        self.matched = torch.empty(R, dtype=torch.int32, device="cuda")
+        self.ids = torch.empty((R, self.mb), dtype=torch.int32, device="cuda")
+        self.ins_ids = torch.empty((R, self.mb), dtype=torch.int32, device="cuda")
+        self.newb = torch.empty(R, dtype=torch.int32, device="cuda")
+        self.nev = torch.zeros(2, dtype=torch.int32, device="cuda")
+        self.h_matched = torch.empty(R, dtype=torch.int32).pin_memory()
+        self.h_ids = torch.empty((R, self.mb), dtype=torch.int32).pin_memory()
+        self.h_newb = torch.empty(R, dtype=torch.int32).pin_memory()
+
+    def step(self, i, e2e=False, events=None):
+        """One pass of the path.  Returns nothing; counters come from ptstore_stats."""
+        torch, G, st = self.torch, self.G, self.store
+        s = self.steps[i]
+        if e2e:
+            d = {k: v.to("cuda", non_blocking=True) for k, v in s["host"].items()}
+        else:
+            d = s["dev"]
+        st.lookup(d["tokens"], d["offsets"], self.mb, G.PIN, self.matched, self.ids)
+        if events is not None:
+            events["fetch"].append((self._ev(), None))
+        st.fetch(self.ids, self.matched, self.cache, d["bt"])
+        if events is not None:
+            events["fetch"][-1] = (events["fetch"][-1][0], self._ev())
+        # the serving engine needs the matched lengths on the host anyway; the same sync gives the free count
+        self.h_matched.copy_(self.matched, non_blocking=True)
+        stats = st.stats()
+        need = s["total_blocks"] - int(self.h_matched.sum())
+        short = need - int(stats.free_blocks[0])
+        if short > 0:
+            st.evict(G.TIER_HBM, short, want_victims=False, n_evicted=self.nev)
+        if events is not None:
+            events["insert"].append((self._ev(), None))
+        st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb)
+        if events is not None:
+            events["insert"][-1] = (events["insert"][-1][0], self._ev())
+        st.release(self.ids, self.matched)
+        if e2e:
+            self.h_ids.copy_(self.ids, non_blocking=True)
+            self.h_newb.copy_(self.newb, non_blocking=True)
+
+    def _ev(self):
+        e = self.torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    def io_bytes(self, i):
+        s = self.steps[i]
+        h2d = sum(v.numel() * v.element_size() for v in s["host"].values())
+        d2h = self.h_matched.numel() * 4 + self.h_ids.numel() * 4 + self.h_newb.numel() * 4
+        return h2d, d2h
+
+
+def run_gpu(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    from __graft_entry__ import build
+    if rank == 0:
+        build()
+    if dist:
+        dist.barrier()
+
+    wl = Llama8BServing(args, rank)
+    n_fill, W_, K = args.fill, args.warmup, args.steps
+    total_steps = n_fill + W_ + K + (W_ + K if not args.no_e2e else 0)
+    wl.prepare(total_steps)
+    block_rw = 2 * wl.sh.block_bytes
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(first, count, e2e, events=None):
+        s0 = wl.store.stats()
+        l0 = wl.store.launch_count()
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for i in range(first, first + count):
+            wl.step(i, e2e=e2e, events=events)
+        t1.record()
+        barrier()
+        ms = t0.elapsed_time(t1)
+        s1 = wl.store.stats()
+        moved = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) + (s1.blocks_inserted - s0.blocks_inserted)
+        return dict(ms=ms, fetched=s1.blocks_fetched[0] - s0.blocks_fetched[0], inserted=s1.blocks_inserted - s0.blocks_inserted,
+                    bytes=moved * block_rw, launches=wl.store.launch_count() - l0,
+                    probes=s1.probes_issued - s0.probes_issued, qblocks=s1.query_blocks - s0.query_blocks,
+                    matched=s1.blocks_matched - s0.blocks_matched, dropped=s1.blocks_dropped[0] - s0.blocks_dropped[0])
+
+    i = 0
+    for _ in range(n_fill + W_):
+        wl.step(i); i += 1
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    events = {"fetch": [], "insert": []}
+    main = timed(i, K, False, events)
+    clocks = sampler.stop() if rank == 0 else None
+    i += K
+    torch.cuda.synchronize()
+    fetch_ms = sum(a.elapsed_time(b) for a, b in events["fetch"])
+    insert_ms = sum(a.elapsed_time(b) for a, b in events["insert"])
+    status = wl.store.status()
+
+    e2e = None
+    if not args.no_e2e:
+        for _ in range(W_):
+            wl.step(i, e2e=True); i += 1
+        e2e = timed(i, K, True)
+        h2d = int(np.mean([wl.io_bytes(j)[0] for j in range(i, i + K)])); d2h = wl.io_bytes(i)[1]
+        i += K
+
+    # aggregate over ranks: max time, sum of bytes
+    def agg(x, op):
+        if not dist:
+            return x
+        t = torch.tensor([float(x)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=op)
+        return float(t.item())
+
+    if dist:
+        MAX, SUM = dist.ReduceOp.MAX, dist.ReduceOp.SUM
+    else:
+        MAX = SUM = None
+    ms = agg(main["ms"], MAX)
+    total_bytes = agg(main["bytes"], SUM)
+    value = total_bytes / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    fetch_bytes = main["fetched"] * block_rw
+    ach = fetch_bytes / (fetch_ms * 1e-3) / 1e9 if fetch_ms > 0 else 0.0
+    out = {
+        "metric": "prefix-hit KV fetch GB/s", "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W_,
+        "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": wl.name, "kv_shape": "32L x 8H x 128 bf16, block 16", "pool_blocks": wl.pool_blocks, "docs": args.docs,
+                   "batch": wl.batch, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
+                   "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
+        "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
+        "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_inserted": main["inserted"] / K, "blocks_dropped": main["dropped"] / K,
+                     "hit_rate_blocks": round(main["matched"] / max(main["qblocks"], 1), 4),
+                     "fetch_call_ms": round(fetch_ms / K, 4), "insert_call_ms": round(insert_ms / K, 4),
+                     "insert_gbps": round(main["inserted"] * block_rw / max(insert_ms, 1e-9) / 1e6, 1),
+                     "lookup_probes": main["probes"] / K},
+        "gpu_launches": int(main["launches"]),
+        "device_status": status,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "copy_%s_kernel<FETCH> (ptstore_fetch)" % args.engine, "achieved": round(ach, 1), "peak": peak,
+                     "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": peak_kind + " (copy, read+write)",
+                     "frac_of_nominal_8TBps": round(ach / NOMINAL_HBM_GBS, 4),
+                     "algorithmic_bytes_per_launch": fetch_bytes / K, "traffic": args.traffic},
+    }
+    if e2e:
+        ems = agg(e2e["ms"], MAX)
+        eb = agg(e2e["bytes"], SUM)
+        out["e2e"] = {"value": round(eb / (ems * 1e-3) / 1e9, 1), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "ms_per_step": round(ems / K, 4)}
+    if rank == 0:
+        if world == 1 and not args.no_cpu:
+            out["cpu_baseline"] = cpu_oracle_sample(args)
+        print(json.dumps(out), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------------------
+def cpu_oracle_sample(args, steps=8, batch=8, pool_blocks=2800):
+    """The CPU oracle, as it stands, on a bounded sample of the same stream: the same step on the same KV
+    shape with `batch` prompts per step and a pool of `pool_blocks` blocks, real bytes moved with memcpy."""
+    from oracle import Oracle, PIN
+    sh = W.LLAMA3_8B
+    stream = W.llama8b_stream(n_docs=args.docs)
+    o = Oracle(sh.layers, sh.heads, sh.dim, sh.elem_bytes, sh.block_tokens, 0, pool_blocks, 0, byte_mode=True)
+    mb = stream.max_blocks
+    B = sh.block_tokens
+    rng = np.random.default_rng(5)
+    batches = [stream.batch(batch)[0] for _ in range(steps + 1)]
+    need_max = max(sum(len(s) // B for s in b) for b in batches)
+    cache = o.new_cache(need_max + 1, fill=3)
+    moved, t_total, probes = 0, 0.0, 0
+    for k, seqs in enumerate(batches):
+        toks, offs = W.ragged(seqs)
+        bt = W.shuffled_block_tables(rng, seqs, B, mb, need_max + 1)
+        t0 = time.perf_counter()
+        m, ids = o.lookup(toks, offs, mb, PIN)
+        o.fetch(ids, m, cache, bt)
+        need = sum(len(s) // B for s in seqs) - int(m.sum())
+        short = need - o.free_count(0)
+        if short > 0:
+            o.evict(0, short, literal=False)
+        ins, newb = o.insert(toks, offs, mb, cache, bt)
+        o.release(ids, m)
+        dt = time.perf_counter() - t0
+        if k == 0:
+            continue                                     # first step only fills the pool
+        t_total += dt
+        moved += (int(m.sum()) + int(newb.sum())) * 2 * sh.block_bytes
+    o.close()
+    return {"value": round(moved / t_total / 1e9, 2), "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": "%d steps of %d prompts of the same document stream, pool %d blocks (%.1f GB), same step sequence; eviction by the "
+                      "sorted closed form" % (steps, batch, pool_blocks, pool_blocks * sh.block_bytes / 1e9),
+            "ms_per_step": round(t_total / steps * 1e3, 1), "host_cores_available": os.cpu_count()}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import build_oracle
+    build_oracle()
+    W_, K = args.warmup, args.steps
+    res = cpu_oracle_sample(args, steps=max(K, 1))
+    out = {"impl": "reference", "metric": "prefix-hit KV fetch GB/s", "value": res["value"], "unit": "GB/s",
+           "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W_, "ms_per_step": res["ms_per_step"],
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+           "config": {"workload": Llama8BServing.name, "note": "CPU oracle on a bounded sample of the workload"},
+           "cpu_baseline": res, "e2e": {"value": res["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--engine", default="bulk", choices=["vector", "bulk"])
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--fill", type=int, default=6, help="untimed steps that fill the pool before warm-up")
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--docs", type=int, default=500)
+    ap.add_argument("--pool-blocks", type=int, default=20000)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per fetch launch, if known (see profiles/)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -56,6 +56,7 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 #define PTSTORE_S_TABLE_FULL  0x2u   /* insert/rebuild: no free slot found within table_slots probes */
 #define PTSTORE_S_BOUNDS      0x4u   /* a block id or block-table entry was out of range; access skipped */
 #define PTSTORE_S_STATE       0x8u   /* release would have driven a refcount below zero; skipped */
+#define PTSTORE_S_TIMEOUT     0x10u  /* a bounded wait inside a copy kernel expired; that CTA stopped copying */
 
 /* flags of ptstore_lookup */
 #define PTSTORE_PIN       0x1u   /* refcount++ on every matched (request, block) pair */
@@ -64,6 +65,11 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 /* flags of ptstore_config_t */
 #define PTSTORE_COPY_VECTOR  0x0u  /* copy engine: 16-byte vector loads/stores (always used for the host tier) */
 #define PTSTORE_COPY_BULK    0x1u  /* copy engine: bulk-async copies through a shared-memory ring (HBM<->HBM) */
+/* tuning fields of flags (0 = library default): lanes per request of the lookup (8, 16 or 32),
+ * copy-kernel variant, copy CTAs per SM */
+#define PTSTORE_LOOKUP_LANES(n)   (((uint32_t)(n) & 0xFFu) << 8)
+#define PTSTORE_COPY_VARIANT(v)   (((uint32_t)(v) & 0xFu) << 16)
+#define PTSTORE_COPY_CTAS_PER_SM(c) (((uint32_t)(c) & 0xFFu) << 20)
 
 /* tiers of ptstore_evict */
 #define PTSTORE_TIER_HBM   0

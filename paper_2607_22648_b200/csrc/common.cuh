@@ -1,0 +1,160 @@
+// Shared device-side definitions of the prefix tensor store: table slot, per-block metadata views,
+// control block, chained block hash.  Everything here is sm_100a device code or POD shared with the
+// host side of the same library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pts {
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+constexpr unsigned FULL = 0xFFFFFFFFu;   // all lanes of a warp
+
+// ---- hash table slot ------------------------------------------------------------------------------
+// 16 bytes, loaded with one 128-bit access.  key 0 = never used, key 1 = deleted.
+// id = NO_ID while a slot has been claimed by an insert that has not assigned its block yet.
+struct __align__(16) Slot {
+  u64 key;
+  u32 id;
+  u32 aux;      // insert only: lowest request index that presented this new key
+};
+constexpr u64 KEY_EMPTY = 0ull;
+constexpr u64 KEY_TOMB = 1ull;
+constexpr u32 NO_ID = 0xFFFFFFFFu;
+constexpr u32 NO_SLOT = 0xFFFFFFFFu;
+
+// ---- status bits / flags (mirror include/ptstore.h) -------------------------------------------------
+constexpr u32 S_NOSPACE = 1u, S_TABLE_FULL = 2u, S_BOUNDS = 4u, S_STATE = 8u, S_TIMEOUT = 16u;
+constexpr u32 F_PIN = 1u, F_NO_TOUCH = 2u;
+
+// ---- control block in device memory ----------------------------------------------------------------
+struct Ring {
+  u32 head;     // position of the next id to hand out
+  u32 count;    // ids available
+};
+struct Ctrl {
+  Ring ring[2];
+  u32 status;
+  u32 pad0;
+  // per-call scalars produced by one kernel and consumed by the next
+  u32 n_pairs;          // fetch / release / insert / demote: entries in the copy descriptor list
+  u32 ins_total_new;    // insert: new unique nodes presented
+  u32 ins_granted;      // insert: of those, how many got a block
+  u32 ins_base;         // insert: ring head before this call
+  u32 ev_want;          // evict: victims still wanted by the current phase
+  u32 ev_cand;          // evict: candidates collected
+  u32 ev_take;          // evict: victims taken by the current phase
+  u32 ev_host_dropped;  // evict: host-tier drops that made room for a demotion
+  u32 live[2];
+  u32 tombstones;
+  u32 pad1;
+  // cumulative counters
+  u64 query_blocks, probes_issued, slots_visited, blocks_matched;
+  u64 blocks_fetched[2];
+  u64 blocks_inserted, blocks_denied;
+  u64 blocks_dropped[2];
+  u64 blocks_demoted;
+  u64 rebuilds;
+};
+
+// ---- everything a kernel needs to know about the store ---------------------------------------------
+struct Store {
+  Slot* table;          // current table
+  u64 slots;
+  // per-block metadata, indexed by block id (both tiers)
+  u64* m_key;           // 0 = block not live
+  u64* m_parent;        // key of the parent node (root key for depth 0)
+  u64* m_last;          // LRU stamp
+  u32* m_ref;
+  u32* m_depth;
+  int* ring_ids[2];
+  u32 n[2];             // blocks per tier
+  Ctrl* ctrl;
+  unsigned char* pool[2];
+  u64 chunk_bytes, block_bytes;
+  u32 layers;
+  u32 block_tokens;
+  u64 root_key;
+};
+
+// ---- chained block hash -----------------------------------------------------------------------------
+// The paper gives each tensor a unique id that an object inherits from its longest common prefix
+// (Section 4.1).  Here the id of a block is a 64-bit key that folds in the key of the parent block,
+// so equal prefixes give equal key sequences and the trie becomes a flat table of keys.
+constexpr u64 HC1 = 0x9E3779B97F4A7C15ull;   // floor(2^64 / golden ratio)
+constexpr u64 HC2 = 0x6A09E667F3BCC909ull;   // frac(sqrt 2) * 2^64, low bit set
+constexpr u64 HC3 = 0xBB67AE8584CAA73Bull;   // frac(sqrt 3) * 2^64
+constexpr u64 HC5 = 0x3C6EF372FE94F82Bull;   // frac(sqrt 5) * 2^64
+
+__host__ __device__ __forceinline__ u64 hmix(u64 x) {
+  x ^= x >> 32; x *= HC3;
+  x ^= x >> 29; x *= HC5;
+  x ^= x >> 32;
+  return x;
+}
+__host__ __device__ __forceinline__ u64 hfix(u64 k) { return k < 2 ? k + 2 : k; }
+__host__ __device__ __forceinline__ u64 hroot(u64 salt) { return hfix(hmix(salt ^ HC2)); }
+__host__ __device__ __forceinline__ u64 hchain(u64 parent, u64 content) { return hfix(hmix(parent * HC1 + content)); }
+__device__ __forceinline__ u64 htoken(int tok, u32 pos) {
+  return hmix((((u64)pos << 32) | (u64)(u32)tok) ^ HC1);
+}
+
+// content hash of one block by ONE thread; 16-byte loads when the block start allows it
+__device__ __forceinline__ u64 content_block(const int* __restrict__ t, u32 B) {
+  u64 s = 0;
+  if (((B & 3u) == 0) && ((reinterpret_cast<uintptr_t>(t) & 15u) == 0)) {
+    const int4* t4 = reinterpret_cast<const int4*>(t);
+    for (u32 j = 0; j < B / 4; ++j) {
+      int4 v = __ldg(t4 + j);
+      s += htoken(v.x, 4 * j) + htoken(v.y, 4 * j + 1) + htoken(v.z, 4 * j + 2) + htoken(v.w, 4 * j + 3);
+    }
+  } else {
+    for (u32 j = 0; j < B; ++j) s += htoken(__ldg(t + j), j);
+  }
+  return s;
+}
+
+// ---- table probing ----------------------------------------------------------------------------------
+__device__ __forceinline__ u64 home_slot(u64 key, u64 slots) { return __umul64hi(key, slots); }
+
+__device__ __forceinline__ Slot load_slot(const Slot* p) {
+  uint4 v = *reinterpret_cast<const uint4*>(p);
+  Slot s;
+  s.key = ((u64)v.y << 32) | v.x;
+  s.id = v.z;
+  s.aux = v.w;
+  return s;
+}
+
+// Linear probe for `key`.  Returns the slot index or NO_SLOT; *visited gets the slots read.
+__device__ __forceinline__ u32 find_slot(const Slot* __restrict__ table, u64 slots, u64 key, u32* visited, u32* id_out) {
+  u64 s = home_slot(key, slots);
+  u32 n = 0;
+  for (u64 i = 0; i < slots; ++i) {
+    Slot v = load_slot(table + s);
+    ++n;
+    if (v.key == key) { *visited = n; *id_out = v.id; return (u32)s; }
+    if (v.key == KEY_EMPTY) break;
+    s = (s + 1 == slots) ? 0 : s + 1;
+  }
+  *visited = n;
+  *id_out = NO_ID;
+  return NO_SLOT;
+}
+
+__device__ __forceinline__ int tier_of(const Store& st, u32 id) { return id < st.n[0] ? 0 : 1; }
+__device__ __forceinline__ unsigned char* block_ptr(const Store& st, u32 id) {
+  return id < st.n[0] ? st.pool[0] + (u64)id * st.block_bytes : st.pool[1] + (u64)(id - st.n[0]) * st.block_bytes;
+}
+
+__device__ __forceinline__ void raise(const Store& st, u32 bit) { atomicOr(&st.ctrl->status, bit); }
+
+// full blocks of request r, capped
+__device__ __forceinline__ int full_blocks(const long long* __restrict__ offsets, int r, u32 B, int max_blocks) {
+  long long len = offsets[r + 1] - offsets[r];
+  long long nb = len < 0 ? 0 : len / (long long)B;
+  return (int)(nb < (long long)max_blocks ? nb : (long long)max_blocks);
+}
+
+}  // namespace pts

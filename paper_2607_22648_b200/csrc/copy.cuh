@@ -1,0 +1,262 @@
+// Copy engine: moves chunks between the store pool and a vLLM-style paged cache (load / store of
+// tensors through application-supplied pointers, paper Section 4.1), or between two pool blocks
+// (flush of owned tensors to a slower tier, Section 4.1 "Access pattern-aware eviction policy").
+//
+// The paper moves all scattered (offset,size) segments of a request "in parallel in a single RDMA RPC"
+// without packing them first (Section 4.1 "RDMA-aware consolidation").  The analogue here is ONE
+// kernel launch over a descriptor list {pool block, cache block}: no staging buffer, every chunk is
+// contiguous on both sides, and a pool block is one contiguous region.
+//
+// Two engines:
+//   vector: every thread moves 16-byte pieces with several independent loads in flight; works for any
+//           device-visible memory (also mapped pinned host memory).
+//   bulk  : one elected thread per CTA drives bulk-async copies global -> shared -> global through a
+//           ring of shared-memory stages tracked by mbarriers; HBM to HBM only.
+// Pure data movement: bounded by HBM bandwidth (or by the host link for the host tier); algorithmic
+// bytes per pool block moved = 2 * block_bytes (read once, write once).
+#pragma once
+#include "common.cuh"
+
+namespace pts {
+
+struct Paged {                 // device view of ptstore_paged_cache_t
+  unsigned char* const* layer_base;
+  u64 kv_stride, block_stride;
+  u32 num_blocks;
+};
+
+enum CopyMode { COPY_FETCH = 0, COPY_INSERT = 1, COPY_POOL = 2 };
+
+// address of piece (ls, off) on both sides of descriptor d
+template <int MODE>
+__device__ __forceinline__ void piece_addr(const Store& st, const Paged& pc, int2 d, u32 ls, u64 off,
+                                           const unsigned char*& src, unsigned char*& dst) {
+  unsigned char* pool_side = block_ptr(st, (u32)d.x) + (u64)ls * st.chunk_bytes + off;
+  if (MODE == COPY_POOL) {
+    src = pool_side;
+    dst = block_ptr(st, (u32)d.y) + (u64)ls * st.chunk_bytes + off;
+  } else {
+    unsigned char* cache_side = pc.layer_base[ls >> 1] + (u64)(ls & 1) * pc.kv_stride + (u64)(u32)d.y * pc.block_stride + off;
+    if (MODE == COPY_FETCH) { src = pool_side; dst = cache_side; }
+    else { src = cache_side; dst = pool_side; }
+  }
+}
+
+__device__ __forceinline__ uint4 ld_stream(const unsigned char* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(unsigned char* p, uint4 v) {
+  asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// ---- vector engine ------------------------------------------------------------------------------------
+// A CTA of THREADS threads moves one piece of THREADS*16*UNROLL bytes per iteration; consecutive CTAs take
+// consecutive pieces, so a pool block is read (or written) front to back by neighbouring CTAs.
+template <int MODE, int THREADS, int UNROLL>
+__global__ void __launch_bounds__(THREADS) copy_vector_kernel(Store st, Paged pc, const int2* __restrict__ desc,
+                                                              const u32* __restrict__ n_pairs_ptr) {
+  constexpr u64 PIECE = (u64)THREADS * 16 * UNROLL;
+  const u32 n_pairs = *n_pairs_ptr;
+  const u32 ppc = (u32)((st.chunk_bytes + PIECE - 1) / PIECE);       // pieces per chunk
+  const u64 per_pair = (u64)2 * st.layers * ppc;
+  const u64 total = (u64)n_pairs * per_pair;
+  for (u64 u = blockIdx.x; u < total; u += gridDim.x) {
+    const u32 pair = (u32)(u / per_pair);
+    const u32 rem = (u32)(u % per_pair);
+    const u32 ls = rem / ppc, piece = rem % ppc;
+    const int2 d = desc[pair];
+    if (d.x < 0) continue;
+    const u64 off = (u64)piece * PIECE;
+    const unsigned char* src;
+    unsigned char* dst;
+    piece_addr<MODE>(st, pc, d, ls, off, src, dst);
+    const u64 left = st.chunk_bytes - off;                           // bytes of this chunk from `off` on
+    uint4 v[UNROLL];
+#pragma unroll
+    for (int k = 0; k < UNROLL; ++k) {
+      const u64 o = ((u64)k * THREADS + threadIdx.x) * 16;
+      if (o < left) v[k] = ld_stream(src + o);
+    }
+#pragma unroll
+    for (int k = 0; k < UNROLL; ++k) {
+      const u64 o = ((u64)k * THREADS + threadIdx.x) * 16;
+      if (o < left) st_stream(dst + o, v[k]);
+    }
+  }
+}
+
+// ---- bulk engine --------------------------------------------------------------------------------------
+__device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
+  u32 ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: gives up after `limit` polls and reports false
+__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, u32 limit) {
+  for (u32 i = 0; i < limit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gsrc, u32 bytes, u64* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* gdst, const void* smem_src, u32 bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr u32 BULK_POLL_LIMIT = 1u << 22;   // polls per wait before the kernel gives up (each poll may suspend briefly)
+
+// One warp per CTA; lane 0 runs the whole pipeline.  STAGES stages of STAGE_BYTES each.
+// Piece p of the launch = pieces p, p+grid, ... ; load of piece i+STAGES-1 is issued once the store of
+// piece i-1 has finished reading its stage, so STAGES-1 loads are in flight per CTA.
+template <int MODE, int STAGES, int STAGE_BYTES>
+__global__ void __launch_bounds__(32) copy_bulk_kernel(Store st, Paged pc, const int2* __restrict__ desc,
+                                                       const u32* __restrict__ n_pairs_ptr) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) u64 bars[STAGES];
+  if (threadIdx.x != 0) return;
+  const u32 n_pairs = *n_pairs_ptr;
+  const u32 ppc = (u32)((st.chunk_bytes + STAGE_BYTES - 1) / STAGE_BYTES);
+  const u64 per_pair = (u64)2 * st.layers * ppc;
+  const u64 total = (u64)n_pairs * per_pair;
+  if (blockIdx.x >= total) return;
+  const u64 mine = (total - blockIdx.x + gridDim.x - 1) / gridDim.x;     // pieces this CTA moves
+
+  for (int s = 0; s < STAGES; ++s) mbar_init(&bars[s], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  fence_async_smem();
+
+  // resolve piece i of this CTA
+  auto resolve = [&](u64 i, const unsigned char*& src, unsigned char*& dst, u32& bytes) -> bool {
+    const u64 u = blockIdx.x + i * gridDim.x;
+    const u32 pair = (u32)(u / per_pair);
+    const u32 rem = (u32)(u % per_pair);
+    const u32 ls = rem / ppc, piece = rem % ppc;
+    const int2 d = desc[pair];
+    if (d.x < 0) return false;
+    const u64 off = (u64)piece * STAGE_BYTES;
+    piece_addr<MODE>(st, pc, d, ls, off, src, dst);
+    const u64 left = st.chunk_bytes - off;
+    bytes = (u32)(left < (u64)STAGE_BYTES ? left : (u64)STAGE_BYTES);
+    return true;
+  };
+  auto issue_load = [&](u64 i) {
+    const unsigned char* src; unsigned char* dst; u32 bytes;
+    const int s = (int)(i % STAGES);
+    if (resolve(i, src, dst, bytes)) {
+      mbar_expect_tx(&bars[s], bytes);
+      bulk_g2s(smem + (size_t)s * STAGE_BYTES, src, bytes, &bars[s]);
+    } else {
+      mbar_expect_tx(&bars[s], 0);            // skipped descriptor: complete the phase with no bytes
+    }
+  };
+
+  const u64 pre = mine < (u64)(STAGES - 1) ? mine : (u64)(STAGES - 1);
+  for (u64 i = 0; i < pre; ++i) issue_load(i);
+  bool ok = true;
+  u64 waited = 0;                              // pieces whose load has been waited for
+  for (u64 i = 0; i < mine; ++i) {
+    const int s = (int)(i % STAGES);
+    const u32 parity = (u32)((i / STAGES) & 1);
+    if (!mbar_wait_bounded(&bars[s], parity, BULK_POLL_LIMIT)) { ok = false; break; }
+    waited = i + 1;
+    const unsigned char* src; unsigned char* dst; u32 bytes;
+    if (resolve(i, src, dst, bytes)) bulk_s2g(dst, smem + (size_t)s * STAGE_BYTES, bytes);
+    bulk_commit();
+    // the stage of piece i-1 is free once its store has read it: at most one newer group may be pending
+    const u64 nxt = i + STAGES - 1;
+    if (nxt < mine) {
+      bulk_wait_read<1>();
+      issue_load(nxt);
+    }
+  }
+  if (!ok) {
+    raise(st, S_TIMEOUT);
+    // drain loads already issued (bounded), so no copy lands in shared memory after exit
+    const u64 issued = (waited + STAGES - 1 < mine) ? waited + STAGES - 1 : mine;
+    for (u64 i = waited; i < issued; ++i)
+      mbar_wait_bounded(&bars[i % STAGES], (u32)((i / STAGES) & 1), BULK_POLL_LIMIT);
+  }
+  bulk_wait_all();
+}
+
+// ---- descriptor lists -----------------------------------------------------------------------------------
+// prefix[r] = sum of min(matched[r'], max_blocks) for r' < r; prefix[R] = total, also stored in ctrl->n_pairs.
+__global__ void __launch_bounds__(1024) scan_matched_kernel(Store st, const int* __restrict__ matched, int R, int max_blocks,
+                                                            u32* __restrict__ prefix) {
+  __shared__ u32 warp_sums[32];
+  __shared__ u32 carry;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < R; base += 1024) {
+    const int r = base + threadIdx.x;
+    int mr = r < R ? matched[r] : 0;
+    mr = mr < 0 ? 0 : (mr > max_blocks ? max_blocks : mr);
+    u32 x = (u32)mr;
+    for (int o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(FULL, x, o); if (lane >= o) x += y; }
+    if (lane == 31) warp_sums[wid] = x;
+    __syncthreads();
+    if (wid == 0) {
+      u32 w = warp_sums[lane];
+      for (int o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(FULL, w, o); if (lane >= o) w += y; }
+      warp_sums[lane] = w;
+    }
+    __syncthreads();
+    const u32 incl = x + (wid ? warp_sums[wid - 1] : 0) + carry;
+    if (r < R) prefix[r] = incl - (u32)mr;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = incl;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { prefix[R] = carry; st.ctrl->n_pairs = carry; }
+}
+
+// desc[prefix[r] + j] = {pool block, cache block} for j < matched[r]; bad entries become {-1,-1}
+__global__ void __launch_bounds__(256) build_pairs_kernel(Store st, const int* __restrict__ ids, const int* __restrict__ matched,
+                                                          const int* __restrict__ bt, int R, int max_blocks, u32 cache_blocks,
+                                                          const u32* __restrict__ prefix, int2* __restrict__ desc) {
+  const long long total = (long long)R * max_blocks;
+  u32 cnt0 = 0, cnt1 = 0;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
+    int mr = matched[r];
+    mr = mr > max_blocks ? max_blocks : mr;
+    if (j >= mr) continue;
+    const int id = ids[e], cb = bt[e];
+    int2 d;
+    if (id < 0 || (u32)id >= st.n[0] + st.n[1] || cb < 0 || (u32)cb >= cache_blocks) {
+      raise(st, S_BOUNDS);
+      d = make_int2(-1, -1);
+    } else {
+      d = make_int2(id, cb);
+      if ((u32)id < st.n[0]) ++cnt0; else ++cnt1;
+    }
+    desc[prefix[r] + j] = d;
+  }
+  cnt0 = __reduce_add_sync(FULL, cnt0);
+  cnt1 = __reduce_add_sync(FULL, cnt1);
+  if ((threadIdx.x & 31) == 0) {
+    if (cnt0) atomicAdd(&st.ctrl->blocks_fetched[0], (u64)cnt0);
+    if (cnt1) atomicAdd(&st.ctrl->blocks_fetched[1], (u64)cnt1);
+  }
+}
+
+}  // namespace pts

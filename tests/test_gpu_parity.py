@@ -1,0 +1,316 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C ABI.
+
+Sizes are small enough for the oracle to finish in seconds but span several copy tiles, several lookup
+chunks and ragged tails.  Everything is integer / byte work: the bar is bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2607_22648_b200 import workloads as W
+
+
+def _imports():
+    from tests.harness import Pair, dev
+    from paper_2607_22648_b200 import binding as G
+    return Pair, dev, G
+
+
+ENGINES = [
+    ("vector", lambda G: G.COPY_VECTOR),
+    ("vector_u8", lambda G: G.COPY_VECTOR | G.copy_variant(1)),
+    ("vector_512", lambda G: G.COPY_VECTOR | G.copy_variant(2)),
+    ("bulk_4x16k", lambda G: G.COPY_BULK),
+    ("bulk_8x8k", lambda G: G.COPY_BULK | G.copy_variant(1)),
+    ("bulk_3x32k", lambda G: G.COPY_BULK | G.copy_variant(2)),
+    ("bulk_6x16k", lambda G: G.COPY_BULK | G.copy_variant(3)),
+]
+
+
+@pytest.mark.parametrize("lanes", [0, 8, 16, 32])
+def test_hash_matches_oracle(lanes):
+    Pair, dev, G = _imports()
+    rng = np.random.default_rng(lanes)
+    for B, shape in [(16, W.TINY), (1, W.KVShape(1, 1, 8, 1)), (3, W.KVShape(1, 2, 8, 3)), (32, W.KVShape(1, 1, 8, 32))]:
+        p = Pair(shape, 16, flags=G.lookup_lanes(lanes), salt=int(rng.integers(0, 1 << 62)), max_requests=64,
+                 max_batch_blocks=64 * 80)
+        seqs = [rng.integers(-5, 32000, size=int(rng.integers(0, 70 * B)), dtype=np.int32) for _ in range(37)]
+        seqs[3] = np.zeros(0, dtype=np.int32)
+        seqs[5] = seqs[4][: max(len(seqs[4]) - 1, 0)]            # unaligned start of the next request
+        for mb in (1, 7, 70, 80):
+            p.hash(seqs, mb)
+        p.close()
+
+
+def tiny_flow(flags, seed=0):
+    Pair, dev, G = _imports()
+    w = W.tiny()
+    sh = w.shape
+    B = sh.block_tokens
+    rng = np.random.default_rng(seed)
+    p = Pair(sh, w.pool_blocks, flags=flags, max_requests=16, max_batch_blocks=16 * 64)
+    smb = W.max_blocks_of(w.store_seqs, B)
+    for i in range(0, len(w.store_seqs), 16):
+        part = w.store_seqs[i:i + 16]
+        need = sum(len(s) // B for s in part)
+        src = W.random_kv_cache(seed * 100 + i, sh, need + 3)
+        bt = W.shuffled_block_tables(rng, part, B, smb, need + 3)
+        p.insert(part, smb, src, bt)
+    assert p.check_status() == 0
+    live = p.check_pools()
+    assert live == p.o.live_count(0) > 300
+    qmb = W.max_blocks_of(w.queries, B)
+    mo, io, _, _ = p.lookup(w.queries, qmb, flags=1)
+    assert mo.max() > 0
+    nd = int(mo.sum()) + 9
+    dst = [np.full((2, nd, sh.chunk_bytes), 0x5A, dtype=np.uint8) for _ in range(sh.layers)]
+    qbt = np.full((len(w.queries), qmb), -1, dtype=np.int32)
+    perm = rng.permutation(nd).astype(np.int32)
+    k = 0
+    for r in range(len(w.queries)):
+        for j in range(mo[r]):
+            qbt[r, j] = perm[k]
+            k += 1
+    p.fetch(io, mo, dst, qbt)
+    p.release(io, mo)
+    assert p.check_status() == 0
+    p.check_counts()
+    return p
+
+
+@pytest.mark.parametrize("name,mk", ENGINES, ids=[e[0] for e in ENGINES])
+def test_tiny_config_insert_lookup_fetch(name, mk):
+    Pair, dev, G = _imports()
+    p = tiny_flow(mk(G))
+    # evict a third, compare victims, look up again
+    ne, v = p.evict(0, 700)
+    assert ne[0] == 700
+    w = W.tiny()
+    p.lookup(w.queries, 64)
+    p.lookup(w.store_seqs[:16], 32)
+    p.check_counts()
+    p.close()
+
+
+def test_insert_dedupe_denial_and_alloc_order():
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 2)
+    p = Pair(sh, 5, max_requests=8, max_batch_blocks=64)
+    a = np.array([1, 1, 2, 2, 3, 3], dtype=np.int32)
+    b = np.array([1, 1, 2, 2, 4, 4, 5, 5], dtype=np.int32)
+    c = np.array([9, 9], dtype=np.int32)
+    rng = np.random.default_rng(0)
+    src = W.random_kv_cache(1, sh, 16)
+    bt = W.shuffled_block_tables(rng, [a, b, a, c], 2, 4, 16)
+    ids, newb = p.insert([a, b, a, c], 4, src, bt)
+    assert ids.tolist() == [[0, 1, 2, -1], [0, 1, 3, 4], [0, 1, 2, -1], [-1, -1, -1, -1]]
+    assert newb.tolist() == [3, 2, 0, 0]
+    assert p.check_status() == G.S_NOSPACE
+    p.check_pools()
+    p.check_counts()
+    # the denied prefix is not findable, the granted ones are
+    mo, io, _, _ = p.lookup([a, b, c], 4)
+    assert mo.tolist() == [3, 4, 0]
+    p.evict(0, 2)
+    p.insert([c, np.array([9, 9, 7, 7, 6, 6], dtype=np.int32)], 4, src, bt[:2])
+    p.check_status()
+    p.check_pools()
+    p.check_counts()
+    p.close()
+
+
+@pytest.mark.parametrize("host", [0, 24])
+def test_random_churn_lockstep(host):
+    """Random interleaving of lookup(PIN) / fetch / evict / insert / release, compared call by call."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(2, 1, 8, 2)
+    B = 2
+    for seed in range(6):
+        rng = np.random.default_rng(100 + seed)
+        p = Pair(sh, 40, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * 12, table_slots=211 if seed % 2 else 401)
+        seqs, pinned = [], []
+        for step in range(60):
+            base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.75 else np.zeros(0, dtype=np.int32)
+            cut = int(rng.integers(0, len(base) + 1))
+            s = np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(1, 10)), dtype=np.int32)])[:24]
+            seqs.append(s)
+            batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(int(rng.integers(1, 5)))] + [s]
+            mb = 12
+            op = rng.random()
+            mo, io, _, _ = p.lookup(batch, mb, flags=1)
+            nd = max(int(mo.sum()), 1) + 2
+            dst = [np.full((2, nd, sh.chunk_bytes), 7, dtype=np.uint8) for _ in range(sh.layers)]
+            bt = np.full((len(batch), mb), -1, dtype=np.int32)
+            perm = rng.permutation(nd)
+            k = 0
+            for r in range(len(batch)):
+                for j in range(mo[r]):
+                    bt[r, j] = perm[k]; k += 1
+            p.fetch(io, mo, dst, bt)
+            if op < 0.7:
+                tier = int(rng.integers(0, 2)) if host else 0
+                p.evict(tier, int(rng.integers(0, 12)), literal=bool(step % 2))
+            need = sum(len(x) // B for x in batch)
+            src = W.random_kv_cache(seed * 1000 + step, sh, need + 1)
+            sbt = W.shuffled_block_tables(rng, batch, B, mb, need + 1)
+            p.insert(batch, mb, src, sbt)
+            if rng.random() < 0.8:
+                p.release(io, mo)
+            else:
+                pinned.append((io, mo))
+            if pinned and rng.random() < 0.3:
+                io2, mo2 = pinned.pop()
+                p.release(io2, mo2)
+            p.check_status()
+            if step % 10 == 9:
+                p.check_pools()
+                p.check_counts()
+        p.check_pools()
+        s = p.check_counts()
+        p.close()
+
+
+def test_lookup_stress_small_matches_oracle():
+    Pair, dev, G = _imports()
+    ws = W.lookup_stress(n_roots=1500, n_queries=2048)
+    sh = W.KVShape(1, 1, 8, 16)
+    for lanes in (8, 16, 32):
+        p = Pair(sh, ws.n_nodes, flags=G.lookup_lanes(lanes), max_requests=2048, max_batch_blocks=2048 * 64,
+                 table_slots=ws.table_slots, byte_mode=False)
+        for i in range(0, len(ws.store_seqs), 2048):
+            p.insert(ws.store_seqs[i:i + 2048], 16)
+        assert p.check_status() == 0
+        mo, io, _, _ = p.lookup(ws.queries, 64)
+        assert (mo == ws.hit_depth).all()
+        p.lookup(ws.queries, 64, flags=3)
+        s = p.check_counts()
+        assert s.live_nodes[0] == ws.n_nodes
+        assert s.query_blocks == 2 * 2048 * 64
+        assert s.blocks_matched == 2 * int(ws.hit_depth.sum())
+        p.release(io, mo)
+        assert p.check_status() == 0
+        p.close()
+
+
+def test_llama8b_shape_fetch_and_insert_span_many_tiles():
+    """2 MiB blocks, 32 KiB chunks: every engine, payload regenerated from tags."""
+    Pair, dev, G = _imports()
+    sh = W.LLAMA3_8B
+    for name, mk in ENGINES:
+        st = W.doc_stream(7, sh, n_docs=6, len_range=(100, 400), zipf_s=1.1, vocab=128256, suffix_range=(5, 40))
+        rng = np.random.default_rng(3)
+        p = Pair(sh, 120, flags=mk(G), max_requests=8, max_batch_blocks=8 * st.max_blocks, byte_mode=False)
+        mb = st.max_blocks
+        wpb = sh.block_bytes // 4
+        g = p.g
+        for step in range(3):
+            seqs, tags = st.batch(5)
+            tm = W.tags_matrix(tags, mb)
+            mo, io, mg, ig = p.lookup(seqs, mb, flags=1)
+            # fetch on the GPU into a device cache; expected content regenerated from the oracle's tags
+            need = sum(len(s) // sh.block_tokens for s in seqs)
+            cache = G.PagedKV(sh.layers, need + 2, sh.chunk_bytes)
+            for t in cache.tensors:
+                t.fill_(0x33)
+            bt = W.shuffled_block_tables(rng, seqs, sh.block_tokens, mb, need + 2)
+            g.fetch(ig, mg, cache, dev(bt))
+            exp_tags = p.o.block_tags(io)
+            for r in range(len(seqs)):
+                for j in range(mo[r]):
+                    want = torch.from_numpy(W.payload_words([exp_tags[r * mb + j]], wpb)).view(torch.uint8).reshape(sh.layers, 2, sh.chunk_bytes)
+                    for l in (0, 13, sh.layers - 1):
+                        got = cache.tensors[l][:, bt[r, j]].cpu()
+                        assert torch.equal(got, want[l]), (name, step, r, j, l)
+            untouched = set(range(need + 2)) - {int(bt[r, j]) for r in range(len(seqs)) for j in range(mo[r])}
+            for b in list(untouched)[:5]:
+                assert bool((cache.tensors[5][:, b] == 0x33).all())
+            # now fill the cache with this batch's payload (as if computed) and insert
+            for r in range(len(seqs)):
+                nb = len(seqs[r]) // sh.block_tokens
+                words = W.payload_words(torch.from_numpy(tm[r, :nb].astype(np.int64)).cuda(), wpb, xp=torch)
+                blk = words.view(torch.uint8).reshape(nb, sh.layers, 2, sh.chunk_bytes)
+                idx = torch.from_numpy(bt[r, :nb].astype(np.int64)).cuda()
+                for l in range(sh.layers):
+                    cache.tensors[l][:, idx] = blk[:, l].permute(1, 0, 2)
+            toks, offs = W.ragged(seqs)
+            io2, no2 = p.o.insert(toks, offs, mb, None, None, tm)
+            ig2, ng2 = g.insert(dev(toks), dev(offs), mb, cache, dev(bt))
+            assert (io2 == ig2.cpu().numpy()).all() and (no2 == ng2.cpu().numpy()).all()
+            p.release(io, mo)
+            # every live pool block holds the payload of its tag
+            pool = g.hbm_pool.view(torch.int32).reshape(g.hbm_blocks, wpb)
+            live = [i for i in range(g.hbm_blocks) if p.o.block_info(i)["live"]]
+            lt = p.o.block_tags(np.array(live, dtype=np.int32))
+            want = W.payload_words(torch.from_numpy(lt.astype(np.int64)).cuda(), wpb, xp=torch)
+            assert torch.equal(pool[torch.tensor(live, device="cuda")], want), (name, step)
+            if step == 1:
+                p.evict(0, 30)
+            p.check_status()
+        p.check_counts()
+        p.close()
+
+
+def test_edge_cases_and_errors():
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 4)
+    p = Pair(sh, 8, max_requests=4, max_batch_blocks=32)
+    g = p.g
+    # empty batch, empty requests, requests shorter than a block
+    z = np.zeros(0, dtype=np.int32)
+    p.lookup([z, z], 4)
+    p.insert([z, np.array([1, 2, 3], dtype=np.int32)], 4)
+    p.hash([z], 4)
+    m, ids = g.lookup(dev(z), dev(np.zeros(1, dtype=np.int64)), 4)
+    assert m.numel() == 0
+    # limits and bad arguments are refused on the host
+    with pytest.raises(G.PTStoreError) as e:
+        g.lookup(dev(z), dev(np.zeros(6, dtype=np.int64)), 4)
+    assert e.value.code == G.E_LIMIT
+    with pytest.raises(G.PTStoreError) as e:
+        g.lookup(dev(z), dev(np.zeros(3, dtype=np.int64)), 0)
+    assert e.value.code == G.E_INVAL
+    with pytest.raises(G.PTStoreError):
+        g.evict(1, 1)                                    # no host tier
+    # out-of-range block table entries and ids are skipped and flagged, nothing else is touched
+    s = np.arange(16, dtype=np.int32)
+    src = W.random_kv_cache(0, sh, 4)
+    p.insert([s], 4, src, np.array([[0, 1, 2, 3]], dtype=np.int32))
+    mo, io, _, _ = p.lookup([s], 4)
+    dst = [np.full((2, 4, sh.chunk_bytes), 9, dtype=np.uint8)]
+    bad_bt = np.array([[0, 7, -3, 1]], dtype=np.int32)
+    p.fetch(io, mo, dst, bad_bt)
+    assert p.check_status() == G.S_BOUNDS
+    bad_ids = io.copy(); bad_ids[0, 1] = 1000
+    p.fetch(bad_ids, mo, dst, np.array([[0, 1, 2, 3]], dtype=np.int32))
+    assert p.check_status() == G.S_BOUNDS
+    # releasing what was never pinned is flagged and leaves counts at zero
+    p.release(io, mo)
+    assert p.check_status() == G.S_STATE
+    ne, v = p.evict(0, 100)
+    assert ne.tolist() == [4, 0]
+    p.check_counts()
+    # max_blocks cap
+    p.insert([s], 2, src, np.array([[0, 1]], dtype=np.int32))
+    mo, io, _, _ = p.lookup([s], 4)
+    assert mo.tolist() == [2]
+    assert g.launch_count() > 10
+    p.close()
+
+
+def test_table_rebuild_under_delete_heavy_churn():
+    """Many evict/insert rounds on a small table: deleted markers pile up, the rebuild reclaims them."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    p = Pair(sh, 64, max_requests=8, max_batch_blocks=8 * 8, table_slots=211)
+    rng = np.random.default_rng(0)
+    for step in range(80):
+        batch = [rng.integers(0, 50, size=8, dtype=np.int32) for _ in range(8)]
+        p.evict(0, 40, literal=False)
+        p.insert(batch, 8)
+        p.lookup(batch, 8)
+        assert p.check_status() == 0
+    s = p.check_counts()
+    assert s.rebuilds > 0
+    p.close()
