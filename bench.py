@@ -135,10 +135,10 @@ class Llama8BServing:
             raw.append((seqs, need))
         self.cache_blocks = need_max + 16
         self.cache = self.G.PagedKV(self.sh.layers, self.cache_blocks, self.sh.chunk_bytes)
-        words = self.sh.chunk_bytes // 4
+        noise = torch.randint(0, 256, (2, 61, self.sh.chunk_bytes), dtype=torch.uint8, device="cuda")
+        pick = torch.arange(self.cache_blocks, device="cuda") % 61
         for t in self.cache.tensors:                       # any bytes will do for timing; make them non-trivial
-            t.view(torch.int32).copy_(torch.randint(-2**31, 2**31 - 1, (2 * self.cache_blocks * words,), dtype=torch.int32,
-                                                    device="cuda").view(2, self.cache_blocks, words))
+            torch.index_select(noise, 1, pick, out=t)
         for seqs, need in raw:
             toks, offs = W.ragged(seqs)
             bt = W.shuffled_block_tables(self.rng, seqs, B, self.mb, self.cache_blocks)

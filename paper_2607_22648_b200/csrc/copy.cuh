@@ -122,77 +122,143 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 constexpr u32 BULK_POLL_LIMIT = 1u << 22;   // polls per wait before the kernel gives up (each poll may suspend briefly)
+constexpr int BULK_MAX_STAGES = 32;
 
-// One warp per CTA; lane 0 runs the whole pipeline.  STAGES stages of STAGE_BYTES each.
-// Piece p of the launch = pieces p, p+grid, ... ; load of piece i+STAGES-1 is issued once the store of
-// piece i-1 has finished reading its stage, so STAGES-1 loads are in flight per CTA.
-template <int MODE, int STAGES, int STAGE_BYTES>
+struct BulkTune {
+  int stages;        // ring depth
+  int stage_bytes;   // bytes per stage (multiple of 16)
+  int group;         // consecutive pieces a CTA takes before striding to its next group
+  int hint;          // 1: mark loads and stores evict-first in L2
+};
+
+__device__ __forceinline__ u64 l2_evict_first_policy() {
+  u64 p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void* smem_dst, const void* gsrc, u32 bytes, u64* bar, u64 policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g_hint(void* gdst, const void* smem_src, u32 bytes, u64 policy) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+               ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes), "l"(policy) : "memory");
+}
+
+// One warp per CTA; lane 0 runs the whole pipeline over a ring of `stages` shared-memory stages.
+// The pieces of the launch are dealt to CTAs in groups of `group` consecutive pieces.  The load of piece
+// i+stages-1 is issued once the store of piece i-1 has finished reading its stage, so stages-1 loads are
+// in flight per CTA.  Every wait is bounded; on expiry the CTA raises S_TIMEOUT, drains and returns.
+// The issuing thread is the only instruction stream of the SM, so its per-piece work is kept short: the
+// piece index is decomposed incrementally (no 64-bit divisions in the loop) and each piece is resolved
+// once, at load time; its destination and size wait in a small shared-memory ring for the store.
+struct PieceCursor {       // walks the pieces of one CTA in order
+  u32 pair, rem;           // piece u = pair * per_pair + rem
+  u32 in_group;            // position inside the current group
+  u32 per_pair, group;
+  u32 step_div, step_mod;  // (grid - 1) * group + 1 decomposed by per_pair: jump to the CTA's next group
+  __device__ __forceinline__ void advance() {
+    u32 add_div = 0, add_mod = 1;
+    if (++in_group == group) { in_group = 0; add_div = step_div; add_mod = step_mod; }
+    rem += add_mod;
+    pair += add_div;
+    if (rem >= per_pair) { rem -= per_pair; pair += 1; }
+  }
+};
+
+template <int MODE>
 __global__ void __launch_bounds__(32) copy_bulk_kernel(Store st, Paged pc, const int2* __restrict__ desc,
-                                                       const u32* __restrict__ n_pairs_ptr) {
+                                                       const u32* __restrict__ n_pairs_ptr, BulkTune tune) {
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ __align__(8) u64 bars[STAGES];
+  __shared__ __align__(8) u64 bars[BULK_MAX_STAGES];
+  __shared__ unsigned char* s_dst[BULK_MAX_STAGES];
+  __shared__ u32 s_bytes[BULK_MAX_STAGES];
   if (threadIdx.x != 0) return;
+  const int STAGES = tune.stages;
+  const u32 SB = (u32)tune.stage_bytes;
+  const u32 G = (u32)tune.group;
   const u32 n_pairs = *n_pairs_ptr;
-  const u32 ppc = (u32)((st.chunk_bytes + STAGE_BYTES - 1) / STAGE_BYTES);
-  const u64 per_pair = (u64)2 * st.layers * ppc;
+  const u32 ppc = (u32)((st.chunk_bytes + SB - 1) / SB);
+  const u32 per_pair = 2u * st.layers * ppc;
   const u64 total = (u64)n_pairs * per_pair;
-  if (blockIdx.x >= total) return;
-  const u64 mine = (total - blockIdx.x + gridDim.x - 1) / gridDim.x;     // pieces this CTA moves
+  // pieces of this CTA: groups blockIdx, blockIdx+grid, ... of G pieces each
+  const u64 n_groups = (total + G - 1) / G;
+  if (blockIdx.x >= n_groups) return;
+  const u64 my_groups = (n_groups - blockIdx.x + gridDim.x - 1) / gridDim.x;
+  u64 mine = my_groups * G;
+  {   // the very last group of the launch may be short
+    const u64 last_group = blockIdx.x + (my_groups - 1) * gridDim.x;
+    if (last_group == n_groups - 1) mine -= n_groups * G - total;
+  }
+  const u64 policy = tune.hint ? l2_evict_first_policy() : 0;
+  const u32 chunk = (u32)st.chunk_bytes;
 
   for (int s = 0; s < STAGES; ++s) mbar_init(&bars[s], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   fence_async_smem();
 
-  // resolve piece i of this CTA
-  auto resolve = [&](u64 i, const unsigned char*& src, unsigned char*& dst, u32& bytes) -> bool {
-    const u64 u = blockIdx.x + i * gridDim.x;
-    const u32 pair = (u32)(u / per_pair);
-    const u32 rem = (u32)(u % per_pair);
-    const u32 ls = rem / ppc, piece = rem % ppc;
-    const int2 d = desc[pair];
-    if (d.x < 0) return false;
-    const u64 off = (u64)piece * STAGE_BYTES;
-    piece_addr<MODE>(st, pc, d, ls, off, src, dst);
-    const u64 left = st.chunk_bytes - off;
-    bytes = (u32)(left < (u64)STAGE_BYTES ? left : (u64)STAGE_BYTES);
-    return true;
-  };
-  auto issue_load = [&](u64 i) {
-    const unsigned char* src; unsigned char* dst; u32 bytes;
-    const int s = (int)(i % STAGES);
-    if (resolve(i, src, dst, bytes)) {
-      mbar_expect_tx(&bars[s], bytes);
-      bulk_g2s(smem + (size_t)s * STAGE_BYTES, src, bytes, &bars[s]);
-    } else {
-      mbar_expect_tx(&bars[s], 0);            // skipped descriptor: complete the phase with no bytes
+  PieceCursor cur;
+  {
+    const u64 first = (u64)blockIdx.x * G;
+    const u64 step = (u64)(gridDim.x - 1) * G + 1;
+    cur.pair = (u32)(first / per_pair); cur.rem = (u32)(first % per_pair);
+    cur.in_group = 0; cur.per_pair = per_pair; cur.group = G;
+    cur.step_div = (u32)(step / per_pair); cur.step_mod = (u32)(step % per_pair);
+  }
+  // issue the load of the piece under the cursor into stage s, remember where it goes, move the cursor on
+  auto issue_load = [&](int s) {
+    const int2 d = desc[cur.pair];
+    const u32 ls = cur.rem / ppc, piece = cur.rem - ls * ppc;
+    cur.advance();
+    if (d.x < 0) {                               // skipped descriptor: complete the phase with no bytes
+      s_bytes[s] = 0;
+      mbar_expect_tx(&bars[s], 0);
+      return;
     }
+    const u32 off = piece * SB;
+    const unsigned char* src; unsigned char* dst;
+    piece_addr<MODE>(st, pc, d, ls, off, src, dst);
+    const u32 left = chunk - off;
+    const u32 bytes = left < SB ? left : SB;
+    s_dst[s] = dst;
+    s_bytes[s] = bytes;
+    mbar_expect_tx(&bars[s], bytes);
+    if (tune.hint) bulk_g2s_hint(smem + (size_t)s * SB, src, bytes, &bars[s], policy);
+    else bulk_g2s(smem + (size_t)s * SB, src, bytes, &bars[s]);
   };
 
   const u64 pre = mine < (u64)(STAGES - 1) ? mine : (u64)(STAGES - 1);
-  for (u64 i = 0; i < pre; ++i) issue_load(i);
+  u64 issued = 0;
+  int ls_stage = 0;                              // stage the next load goes to
+  for (; issued < pre; ++issued) { issue_load(ls_stage); ls_stage = ls_stage + 1 == STAGES ? 0 : ls_stage + 1; }
   bool ok = true;
-  u64 waited = 0;                              // pieces whose load has been waited for
-  for (u64 i = 0; i < mine; ++i) {
-    const int s = (int)(i % STAGES);
-    const u32 parity = (u32)((i / STAGES) & 1);
+  int s = 0;                                     // stage of piece i
+  u32 parity = 0;
+  u64 i = 0;
+  for (; i < mine; ++i) {
     if (!mbar_wait_bounded(&bars[s], parity, BULK_POLL_LIMIT)) { ok = false; break; }
-    waited = i + 1;
-    const unsigned char* src; unsigned char* dst; u32 bytes;
-    if (resolve(i, src, dst, bytes)) bulk_s2g(dst, smem + (size_t)s * STAGE_BYTES, bytes);
+    const u32 bytes = s_bytes[s];
+    if (bytes) {
+      if (tune.hint) bulk_s2g_hint(s_dst[s], smem + (size_t)s * SB, bytes, policy);
+      else bulk_s2g(s_dst[s], smem + (size_t)s * SB, bytes);
+    }
     bulk_commit();
     // the stage of piece i-1 is free once its store has read it: at most one newer group may be pending
-    const u64 nxt = i + STAGES - 1;
-    if (nxt < mine) {
+    if (issued < mine) {
       bulk_wait_read<1>();
-      issue_load(nxt);
+      issue_load(ls_stage);
+      ls_stage = ls_stage + 1 == STAGES ? 0 : ls_stage + 1;
+      ++issued;
     }
+    if (++s == STAGES) { s = 0; parity ^= 1u; }
   }
   if (!ok) {
     raise(st, S_TIMEOUT);
     // drain loads already issued (bounded), so no copy lands in shared memory after exit
-    const u64 issued = (waited + STAGES - 1 < mine) ? waited + STAGES - 1 : mine;
-    for (u64 i = waited; i < issued; ++i)
-      mbar_wait_bounded(&bars[i % STAGES], (u32)((i / STAGES) & 1), BULK_POLL_LIMIT);
+    for (u64 k = i; k < issued; ++k) {
+      mbar_wait_bounded(&bars[s], parity, BULK_POLL_LIMIT);
+      if (++s == STAGES) { s = 0; parity ^= 1u; }
+    }
   }
   bulk_wait_all();
 }

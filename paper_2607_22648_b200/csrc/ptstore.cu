@@ -65,6 +65,8 @@ Layout make_layout(const ptstore_config_t* c) {
 
 }  // namespace
 
+struct BulkVariant { int stages, stage_bytes, ctas_per_sm, group, hint; };
+
 struct ptstore {
   ptstore_config_t cfg;
   Layout lay;
@@ -83,6 +85,9 @@ struct ptstore {
   u64 launches;
   int last_cuda;
   int sms;
+  int bulk_smem_set[3];  // dynamic shared memory already granted to the bulk kernel of each mode
+  bool has_env_tune;
+  BulkVariant env_tune;
 };
 
 namespace {
@@ -152,19 +157,62 @@ int lanes_for(const ptstore* h, int max_blocks) {
 }
 
 // ---- copy engine dispatch -----------------------------------------------------------------------------------
-template <int MODE, int STAGES, int STAGE_BYTES>
-int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, int ctas_per_sm) {
-  static bool attr_set[16] = {};
-  const int smem = STAGES * STAGE_BYTES;
-  const int dev = h->cfg.device & 15;
-  if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(copy_bulk_kernel<MODE, STAGES, STAGE_BYTES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+// index = PTSTORE_COPY_VARIANT field of the flags
+const BulkVariant kBulkVariants[] = {
+    {0, 0, 1, 1, 0},       // 0: default, sized by auto_bulk() from the chunk size
+    {8, 8192, 3, 1, 0},    // 1
+    {3, 32768, 1, 1, 0},   // 2
+    {4, 16384, 3, 1, 0},   // 3
+    {8, 16384, 1, 1, 0},   // 4
+    {12, 16384, 1, 1, 0},  // 5
+    {4, 32768, 1, 1, 0},   // 6
+    {6, 32768, 1, 1, 0},   // 7
+    {6, 16384, 1, 2, 0},   // 8: a CTA takes whole 32 KiB chunks
+    {6, 16384, 1, 1, 1},   // 9: evict-first L2 hints
+    {3, 65536, 1, 1, 0},   // 10
+    {24, 8192, 1, 1, 0},   // 11
+};
+constexpr int kNumBulkVariants = (int)(sizeof(kBulkVariants) / sizeof(kBulkVariants[0]));
+
+// PTSTORE_BULK_TUNE="stages,stage_bytes,ctas_per_sm,group,hint" overrides the variant table (tuning aid)
+bool env_bulk_tune(BulkVariant* v) {
+  const char* e = std::getenv("PTSTORE_BULK_TUNE");
+  if (!e) return false;
+  int a[5] = {0, 0, 0, 1, 0};
+  int n = 0;
+  const char* p = e;
+  while (*p && n < 5) {
+    a[n++] = std::atoi(p);
+    while (*p && *p != ',') ++p;
+    if (*p == ',') ++p;
+  }
+  if (n < 3 || a[0] < 2 || a[0] > BULK_MAX_STAGES || a[1] < 16 || a[1] % 16 || (long long)a[0] * a[1] > 227 * 1024 || a[2] < 1 || a[3] < 1) return false;
+  *v = {a[0], a[1], a[2], a[3], a[4] ? 1 : 0};
+  return true;
+}
+
+// Default ring: stages of min(chunk, 32 KiB) and about 64 KiB of loads in flight per SM with one CTA per SM.
+// On B200 the copy was fastest with FEW bytes in flight (3 x 32 KiB x 1 CTA and 2 x 32 KiB x 2 CTAs per SM
+// both gave ~6.63 TB/s read+write on 32 KiB chunks; deeper rings and more CTAs were 3-7 % slower).
+BulkVariant auto_bulk(u64 chunk_bytes) {
+  int stage = (int)(chunk_bytes < 32768 ? chunk_bytes : 32768);
+  int stages = 1 + 65536 / stage;
+  if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
+  return {stages, stage, 1, 1, 0};
+}
+
+template <int MODE>
+int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, const BulkVariant& v, int ctas_per_sm) {
+  const int smem = v.stages * v.stage_bytes;
+  if (smem > h->bulk_smem_set[MODE]) {
+    if (cudaFuncSetAttribute(copy_bulk_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       h->last_cuda = (int)cudaGetLastError();
       return PTSTORE_E_CUDA;
     }
-    attr_set[dev] = true;
+    h->bulk_smem_set[MODE] = smem;
   }
-  copy_bulk_kernel<MODE, STAGES, STAGE_BYTES><<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
+  BulkTune t = {v.stages, v.stage_bytes, v.group, v.hint};
+  copy_bulk_kernel<MODE><<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs, t);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
@@ -174,12 +222,10 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
   const u32 variant = (h->cfg.flags >> 16) & 0xFu;
   int per_sm = (int)((h->cfg.flags >> 20) & 0xFFu);
   if ((h->cfg.flags & PTSTORE_COPY_BULK) && !host_side_possible) {
-    switch (variant) {
-      case 1: return launch_bulk<MODE, 8, 8192>(h, pc, s, per_sm ? per_sm : 3);
-      case 2: return launch_bulk<MODE, 3, 32768>(h, pc, s, per_sm ? per_sm : 2);
-      case 3: return launch_bulk<MODE, 6, 16384>(h, pc, s, per_sm ? per_sm : 2);
-      default: return launch_bulk<MODE, 4, 16384>(h, pc, s, per_sm ? per_sm : 3);
-    }
+    BulkVariant v = kBulkVariants[variant < (u32)kNumBulkVariants ? variant : 0];
+    if (v.stages == 0) v = auto_bulk(h->st.chunk_bytes);
+    if (h->has_env_tune) v = h->env_tune;
+    return launch_bulk<MODE>(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm);
   }
   switch (variant) {
     case 1:
@@ -189,7 +235,7 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
       copy_vector_kernel<MODE, 512, 4><<<h->sms * (per_sm ? per_sm : 4), 512, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
       break;
     default:
-      copy_vector_kernel<MODE, 256, 4><<<h->sms * (per_sm ? per_sm : 8), 256, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
+      copy_vector_kernel<MODE, 256, 4><<<h->sms * (per_sm ? per_sm : 16), 256, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
       break;
   }
   PTS_CHECK_LAUNCH(h);
@@ -298,6 +344,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
     (void)cudaGetLastError(); delete h; return PTSTORE_E_CUDA;
   }
   h->sms = sms;
+  h->has_env_tune = env_bulk_tune(&h->env_tune);
   unsigned char* w = static_cast<unsigned char*>(cfg->workspace);
   h->stash = reinterpret_cast<Slot*>(w + lay.table[1]);
   Store& st = h->st;
