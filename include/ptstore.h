@@ -228,6 +228,30 @@ uint64_t ptstore_launch_count(const ptstore_t* st);
 /* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
 int ptstore_last_cuda_error(const ptstore_t* st);
 
+/*
+ * Gather without a handle, a workspace or any allocation (the paper has no counterpart: its store always
+ * owns an allocator, Section 5).  For callers that must not call cudaMalloc — code running after a
+ * serving engine has frozen its memory budget, or a plugin that receives pointers but no allocator — and
+ * therefore cannot supply the workspace a handle needs.  Does exactly what ptstore_fetch does for HBM
+ * block ids: for every r, j < matched_blocks[r], layer and K/V plane, one chunk is copied from pool
+ * block block_ids[r*max_blocks+j] to cache block block_tables[r*max_blocks+j].
+ *   hbm_pool     device memory, [hbm_blocks][num_layers][2][chunk_bytes], 16-byte aligned
+ *   status_out   device uint32 or NULL: receives PTSTORE_S_BOUNDS if an id or table entry was skipped, else 0
+ * Scratch (prefix sums, descriptor list) is a fixed device array inside the library, PTSTORE_STATIC_SCRATCH_BYTES
+ * on every GPU that loads it, held until process exit.  Limits: R <= PTSTORE_STATIC_MAX_REQUESTS and
+ * R*max_blocks <= PTSTORE_STATIC_MAX_PAIRS, else PTSTORE_E_LIMIT.  All calls on a GPU share that array: calls
+ * that overlap on the GPU race, so keep them on one stream or order them.  The first call on each device
+ * (made with that device current) looks up the array's address; issue it before any stream capture.
+ * Calls no cudaMalloc / cudaFree / allocating routine.  Enqueues on `stream` and returns.
+ */
+#define PTSTORE_STATIC_MAX_REQUESTS   1024u
+#define PTSTORE_STATIC_MAX_PAIRS      65536u
+#define PTSTORE_STATIC_SCRATCH_BYTES  (1024u + 4352u + 8u * PTSTORE_STATIC_MAX_PAIRS)
+int ptstore_fetch_static(const void* hbm_pool, uint32_t hbm_blocks, uint32_t num_layers, uint64_t chunk_bytes,
+                         const int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
+                         const ptstore_paged_cache_t* dst /*host struct*/, const int32_t* block_tables,
+                         uint32_t* status_out, ptstore_stream_t stream);
+
 /* Static text for a PTSTORE_E_* code. */
 const char* ptstore_strerror(int code);
 

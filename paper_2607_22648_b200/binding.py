@@ -55,7 +55,7 @@ class Stats(C.Structure):
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
-           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror"]
+           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static"]
 
 
 def _load():
@@ -79,6 +79,7 @@ def _load():
     lib.ptstore_launch_count.restype = u64
     lib.ptstore_launch_count.argtypes = [vp]
     lib.ptstore_last_cuda_error.argtypes = [vp]
+    lib.ptstore_fetch_static.argtypes = [vp, u32, u32, u64, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp]
     lib.ptstore_strerror.restype = C.c_char_p
     lib.ptstore_strerror.argtypes = [C.c_int]
     return lib
@@ -113,6 +114,21 @@ class PagedKV:
         t0 = self.tensors[0]
         self.desc = PagedCache(self.ptrs.data_ptr(), t0.stride(0) * t0.element_size(), t0.stride(1) * t0.element_size(),
                                num_blocks, 0)
+
+
+STATIC_MAX_REQUESTS, STATIC_MAX_PAIRS = 1024, 65536
+
+
+def fetch_static(hbm_pool, hbm_blocks, layers, chunk_bytes, ids, matched, cache, block_tables, status_out=None):
+    """ptstore_fetch_static: the gather for callers that may not allocate device memory.  Needs no store
+    handle; scratch is a fixed array inside the library (limits STATIC_MAX_REQUESTS / STATIC_MAX_PAIRS).
+    Calls that overlap on the GPU race on that array; the first call per device should precede any stream
+    capture.  Raises PTStoreError on a refused call."""
+    R, mb = ids.shape
+    rc = lib.ptstore_fetch_static(_ptr(hbm_pool), hbm_blocks, layers, chunk_bytes, _ptr(ids), _ptr(matched), R, mb,
+                                  C.byref(cache.desc), _ptr(block_tables), _ptr(status_out), _stream())
+    if rc:
+        raise PTStoreError(rc, "ptstore_fetch_static")
 
 
 class PTStore:
