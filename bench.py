@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 from paper_2607_22648_b200 import workloads as W  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per block moved by the fetch copy kernel, from the ncu capture of a small case (profiles/): traffic grows in
+# proportion to the blocks moved, so a full launch is this figure times its blocks.
+NCU_DRAM_BYTES_PER_FETCHED_BLOCK = (1.153515e9 + 1.109151e9) / 529
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -308,7 +311,9 @@ def run_gpu(args):
         "roofline": {"bound": "hbm", "kernel": "copy_%s_kernel<FETCH> (ptstore_fetch)" % args.engine, "achieved": round(ach, 1), "peak": peak,
                      "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": peak_kind + " (copy, read+write)",
                      "frac_of_nominal_8TBps": round(ach / NOMINAL_HBM_GBS, 4),
-                     "algorithmic_bytes_per_launch": fetch_bytes / K, "traffic": args.traffic},
+                     "algorithmic_bytes_per_launch": fetch_bytes / K,
+                     "traffic": args.traffic if args.traffic else round(NCU_DRAM_BYTES_PER_FETCHED_BLOCK * main["fetched"] / K),
+                     "traffic_kind": "ncu DRAM read+write bytes of a 529-block launch scaled by blocks moved"},
     }
     if e2e:
         ems = agg(e2e["ms"], MAX)
