@@ -1,0 +1,128 @@
+"""Full-size parity on the GPU: the workloads at their stated sizes, in the launch configuration the bench
+times (bulk copy engine, default ring), against the CPU oracle in tag mode.
+
+All integer outputs are compared exhaustively; K/V bytes against payload regenerated from the oracle's
+tags (every fetched block on the GPU, plus >= 256 sampled chunks byte for byte on the host).  Sizes shrink
+only if the device or host cannot hold them, and the test prints the size it used.
+"""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2607_22648_b200 import workloads as W
+
+
+def _free_gb():
+    import gc
+    gc.collect()
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()                   # earlier tests in this process must not shrink these sizes
+    free, total = torch.cuda.mem_get_info()
+    return free / 1e9
+
+
+def test_llama8b_pool20k_batch64_serving_steps():
+    """config 2 at full size: 20,000-block pool (39 GiB), 500 documents, 64 prompts per step."""
+    from tests.serving import LockstepServing
+    sh = W.LLAMA3_8B
+    pool = 20000 if _free_gb() > 100 else 6000
+    st = W.llama8b_stream()
+    mb = st.max_blocks
+    batches = [st.batch(64) for _ in range(5)]
+    cache_blocks = max(sum(len(s) // sh.block_tokens for s in b[0]) for b in batches) + 8
+    srv = LockstepServing(sh, pool, 0, 64, mb, cache_blocks, seed=2)
+    seen_evict = False
+    for k, (seqs, tags) in enumerate(batches):
+        r = srv.step(seqs, tags, sample=80, check_all=True, poison=(k == 3))
+        seen_evict |= r["evicted"] is not None
+        assert r["status"] == 0
+    s = srv.check_counts()
+    assert srv.check_pool(48) > 0
+    assert seen_evict and s.free_blocks[0] < 64 * mb
+    assert srv.sampled_chunks >= 256 and srv.checked_blocks > 20000
+    print("llama8b full size: pool %d blocks, fetched blocks checked %d, sampled chunks %d" % (pool, srv.checked_blocks, srv.sampled_chunks))
+    srv.close()
+
+
+def test_lookup_stress_one_million_nodes():
+    """config 3 at full size: 10^6-node trie at load factor 0.7, 16,384 requests x 64 blocks."""
+    from tests.harness import Pair, dev
+    from paper_2607_22648_b200 import binding as G
+    ws = W.lookup_stress()
+    assert ws.n_nodes == 1000000 and ws.table_slots == 1428572
+    sh = W.KVShape(1, 1, 8, 16)
+    p = Pair(sh, ws.n_nodes, max_requests=16384, max_batch_blocks=16384 * 64, table_slots=ws.table_slots, byte_mode=False)
+    for i in range(0, len(ws.store_seqs), 8192):
+        p.insert(ws.store_seqs[i:i + 8192], 16)
+    assert p.check_status() == 0
+    mo, io, _, _ = p.lookup(ws.queries, 64)
+    assert (mo == ws.hit_depth).all()
+    assert 5.0 < mo.mean() < 8.0
+    mo2, io2, _, _ = p.lookup(ws.queries, 64, flags=G.PIN | G.NO_TOUCH)
+    s = p.check_counts()
+    assert s.live_nodes[0] == 1000000 and s.free_blocks[0] == 0
+    assert s.query_blocks == 2 * 16384 * 64 and s.blocks_matched == 2 * int(mo.sum())
+    # probes are issued a chunk of blocks at a time, so at least one per matched block plus the terminating miss
+    assert 2 * int(mo.sum()) <= s.probes_issued <= s.query_blocks
+    p.release(io2, mo2)
+    assert p.check_status() == 0
+    # all-hit variant: queries are stored paths, no early stop
+    wa = W.lookup_stress(all_hit=True, n_queries=4096)
+    ma, ia, _, _ = p.lookup(wa.queries, 64)
+    assert (ma == wa.hit_depth).all() and ma.min() >= 5
+    print("lookup stress: mean hit depth %.2f, slots visited per probe %.3f" % (mo.mean(), s.slots_visited / max(s.probes_issued, 1)))
+    p.close()
+
+
+def test_llama70b_16k_prefix_fetch_shuffled_tables():
+    """config 4: 80 layers, 32-token blocks (10 MiB), 16k-token documents, batch of 8."""
+    from tests.serving import LockstepServing
+    sh = W.LLAMA3_70B
+    st = W.llama70b_stream()
+    mb = st.max_blocks                                     # 513
+    cache_blocks = 8 * mb
+    # pool ~100 GB if the device can hold pool + 43 GB of paged cache, else what fits
+    budget = _free_gb() - cache_blocks * sh.block_bytes / 1e9 - 6
+    pool = int(min(9536, budget * 1e9 // sh.block_bytes))
+    assert pool >= 3 * 513, "device too small for this test"
+    srv = LockstepServing(sh, pool, 0, 8, mb, cache_blocks, seed=4)
+    for k in range(4):
+        seqs, tags = st.batch(8)
+        r = srv.step(seqs, tags, sample=100, check_all=(k >= 2), poison=(k == 3))
+    assert r["matched"] >= 4 * 512                          # Zipf(1.2) over 18 documents: most of the batch hits
+    srv.check_counts()
+    assert srv.check_pool(8) > 0
+    assert srv.sampled_chunks >= 256
+    print("llama70b: pool %d blocks (%.1f GB), last step matched %d of %d blocks" % (pool, pool * sh.block_bytes / 1e9, r["matched"], r["total"]))
+    srv.close()
+
+
+def test_churn_with_host_tier():
+    """config 5: Llama-3-8B shape, 40 GB HBM store + pinned-host store, Zipf(1.0) over 5000 documents,
+    micro-batches of 16 with LRU demotion to the host tier and drops from it."""
+    import psutil
+    from tests.serving import LockstepServing
+    sh = W.LLAMA3_8B
+    st = W.churn_stream()
+    mb = st.max_blocks
+    hbm = 19073 if _free_gb() > 80 else 4000
+    host_gb = min(200.0, psutil.virtual_memory().available / 1e9 * 0.35)
+    host = int(host_gb * 1e9 // sh.block_bytes)
+    cache_blocks = 16 * mb
+    srv = LockstepServing(sh, hbm, host, 16, mb, cache_blocks, seed=5)
+    n_steps = 60
+    demoted = dropped = 0
+    for k in range(n_steps):
+        seqs, tags = st.batch(16)
+        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9))
+        if r["evicted"] is not None:
+            demoted += int(r["evicted"][0]); dropped += int(r["evicted"][1])
+    s = srv.check_counts()
+    assert srv.check_pool(32) > 0
+    assert demoted > 0 and s.blocks_demoted == demoted
+    assert srv.sampled_chunks >= 256
+    print("churn: hbm %d blocks, host %d blocks (%.0f GB pinned), %d steps, demoted %d, host drops %d, fetched from hbm/host %s"
+          % (hbm, host, host * sh.block_bytes / 1e9, n_steps, demoted, dropped, srv.fetched_by_tier))
+    srv.close()
