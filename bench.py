@@ -106,22 +106,45 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------------------
-class Llama8BServing:
-    """configs[1]: the workload the metric is quoted on."""
-    name = "llama3_8b_kv_pool20k_zipf1.1_batch64"
+class Serving:
+    """Serving-loop workloads: llama8b = configs[1] (the one the metric is quoted on), llama70b = configs[3],
+    churn = configs[4] (HBM + pinned-host tiers)."""
 
-    def __init__(self, args, rank):
+    def __init__(self, args, rank, kind="llama8b"):
         import torch
         from paper_2607_22648_b200 import binding as G
-        self.torch, self.G = torch, G
-        self.sh = W.LLAMA3_8B
-        self.batch, self.pool_blocks = args.batch, args.pool_blocks
-        self.stream = W.llama8b_stream(seed=W.BASE_SEED + 1 + 1000 * rank, n_docs=args.docs)
+        self.torch, self.G, self.kind = torch, G, kind
+        free_gb = torch.cuda.mem_get_info()[0] / 1e9
+        host_blocks = 0
+        if kind == "llama8b":
+            self.sh = W.LLAMA3_8B
+            self.batch, self.pool_blocks = args.batch or 64, args.pool_blocks or 20000
+            self.stream = W.llama8b_stream(seed=W.BASE_SEED + 1 + 1000 * rank, n_docs=args.docs or 500)
+            self.name = "llama3_8b_kv_pool%dk_zipf1.1_batch%d" % (self.pool_blocks // 1000, self.batch)
+            self.kv = "32L x 8H x 128 bf16, block 16"
+        elif kind == "llama70b":
+            self.sh = W.LLAMA3_70B
+            self.batch = args.batch or 8
+            self.stream = W.llama70b_stream(seed=W.BASE_SEED + 3 + 1000 * rank, n_docs=args.docs or 18)
+            cache_gb = self.batch * self.stream.max_blocks * self.sh.block_bytes / 1e9
+            self.pool_blocks = args.pool_blocks or int(min(9536, (free_gb - cache_gb - 8) * 1e9 // self.sh.block_bytes))
+            self.name = "llama3_70b_kv_pool%d_zipf1.2_batch%d_16k_prefix" % (self.pool_blocks, self.batch)
+            self.kv = "80L x 8H x 128 bf16, block 32"
+        else:
+            import psutil
+            self.sh = W.LLAMA3_8B
+            self.batch, self.pool_blocks = args.batch or 16, args.pool_blocks or 19073
+            self.stream = W.churn_stream(seed=W.BASE_SEED + 4 + 1000 * rank, n_docs=args.docs or 5000)
+            host_gb = args.host_gb if args.host_gb else min(200.0, psutil.virtual_memory().available / 1e9 * 0.4)
+            host_blocks = int(host_gb * 1e9 // self.sh.block_bytes)
+            self.name = "churn_llama3_8b_kv_hbm%d_host%d_zipf1.0_batch%d" % (self.pool_blocks, host_blocks, self.batch)
+            self.kv = "32L x 8H x 128 bf16, block 16"
+        self.host_blocks = host_blocks
         self.mb = self.stream.max_blocks
         flags = (G.COPY_BULK if args.engine == "bulk" else G.COPY_VECTOR) | G.copy_variant(args.variant) | \
             G.copy_ctas_per_sm(args.ctas_per_sm)
         self.store = G.PTStore(self.sh.layers, self.sh.heads, self.sh.dim, self.sh.block_tokens, self.pool_blocks,
-                               max_requests=self.batch, max_batch_blocks=self.batch * self.mb, flags=flags)
+                               max_requests=self.batch, max_batch_blocks=self.batch * self.mb, flags=flags, host_blocks=host_blocks)
         self.rng = np.random.default_rng(W.BASE_SEED + 77 + rank)
         self.steps = []
         self.cache = None
@@ -180,7 +203,11 @@ class Llama8BServing:
         need = s["total_blocks"] - int(self.h_matched.sum())
         short = need - int(stats.free_blocks[0])
         if short > 0:
+            if events is not None:
+                events["evict"].append((self._ev(), None))
             st.evict(G.TIER_HBM, short, want_victims=False, n_evicted=self.nev)
+            if events is not None:
+                events["evict"][-1] = (events["evict"][-1][0], self._ev())
         if events is not None:
             events["insert"].append((self._ev(), None))
         st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb)
@@ -221,7 +248,7 @@ def run_gpu(args):
     if dist:
         dist.barrier()
 
-    wl = Llama8BServing(args, rank)
+    wl = Serving(args, rank, args.workload)
     n_fill, W_, K = args.fill, args.warmup, args.steps
     total_steps = n_fill + W_ + K + (W_ + K if not args.no_e2e else 0)
     wl.prepare(total_steps)
@@ -245,8 +272,11 @@ def run_gpu(args):
         barrier()
         ms = t0.elapsed_time(t1)
         s1 = wl.store.stats()
-        moved = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) + (s1.blocks_inserted - s0.blocks_inserted)
-        return dict(ms=ms, fetched=s1.blocks_fetched[0] - s0.blocks_fetched[0], inserted=s1.blocks_inserted - s0.blocks_inserted,
+        fetched = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) + (s1.blocks_fetched[1] - s0.blocks_fetched[1])
+        moved = fetched + (s1.blocks_inserted - s0.blocks_inserted) + (s1.blocks_demoted - s0.blocks_demoted)
+        return dict(ms=ms, fetched=fetched, fetched_host=s1.blocks_fetched[1] - s0.blocks_fetched[1],
+                    inserted=s1.blocks_inserted - s0.blocks_inserted, demoted=s1.blocks_demoted - s0.blocks_demoted,
+                    host_dropped=s1.blocks_dropped[1] - s0.blocks_dropped[1],
                     bytes=moved * block_rw, launches=wl.store.launch_count() - l0,
                     probes=s1.probes_issued - s0.probes_issued, qblocks=s1.query_blocks - s0.query_blocks,
                     matched=s1.blocks_matched - s0.blocks_matched, dropped=s1.blocks_dropped[0] - s0.blocks_dropped[0])
@@ -257,13 +287,14 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    events = {"fetch": [], "insert": []}
+    events = {"fetch": [], "insert": [], "evict": []}
     main = timed(i, K, False, events)
     clocks = sampler.stop() if rank == 0 else None
     i += K
     torch.cuda.synchronize()
     fetch_ms = sum(a.elapsed_time(b) for a, b in events["fetch"])
     insert_ms = sum(a.elapsed_time(b) for a, b in events["insert"])
+    evict_ms = sum(a.elapsed_time(b) for a, b in events["evict"])
     status = wl.store.status()
 
     e2e = None
@@ -296,7 +327,7 @@ def run_gpu(args):
         "metric": "prefix-hit KV fetch GB/s", "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W_,
         "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8", "data": "synthetic",
-        "config": {"workload": wl.name, "kv_shape": "32L x 8H x 128 bf16, block 16", "pool_blocks": wl.pool_blocks, "docs": args.docs,
+        "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(wl.stream.docs),
                    "batch": wl.batch, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
                    "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
@@ -304,20 +335,25 @@ def run_gpu(args):
                      "hit_rate_blocks": round(main["matched"] / max(main["qblocks"], 1), 4),
                      "fetch_call_ms": round(fetch_ms / K, 4), "insert_call_ms": round(insert_ms / K, 4),
                      "insert_gbps": round(main["inserted"] * block_rw / max(insert_ms, 1e-9) / 1e6, 1),
-                     "lookup_probes": main["probes"] / K},
+                     "lookup_probes": main["probes"] / K, "blocks_fetched_from_host": main["fetched_host"] / K,
+                     "blocks_demoted": main["demoted"] / K, "host_blocks_dropped": main["host_dropped"] / K,
+                     "evict_call_ms": round(evict_ms / K, 4),
+                     "demote_gbps_one_way": round(main["demoted"] * wl.sh.block_bytes / max(evict_ms, 1e-9) / 1e6, 1)},
         "gpu_launches": int(main["launches"]),
         "device_status": status,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "copy_%s_kernel<FETCH> (ptstore_fetch)" % args.engine, "achieved": round(ach, 1), "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "copy_%s_kernel<FETCH> (ptstore_fetch)" % ("vector" if wl.host_blocks else args.engine), "achieved": round(ach, 1), "peak": peak,
                      "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": peak_kind + " (copy, read+write)",
                      "frac_of_nominal_8TBps": round(ach / NOMINAL_HBM_GBS, 4),
                      "algorithmic_bytes_per_launch": fetch_bytes / K,
-                     "traffic": args.traffic if args.traffic else round(NCU_DRAM_BYTES_PER_FETCHED_BLOCK * main["fetched"] / K),
+                     "traffic": args.traffic if args.traffic else round(NCU_DRAM_BYTES_PER_FETCHED_BLOCK / (2 * W.LLAMA3_8B.block_bytes) * fetch_bytes / K),
                      "traffic_kind": "ncu DRAM read+write bytes of a 529-block launch scaled by blocks moved"},
     }
     if e2e:
         ems = agg(e2e["ms"], MAX)
         eb = agg(e2e["bytes"], SUM)
+        if wl.host_blocks:
+            out["host_link_gbps_measured"] = host_link_gbps(torch)
         out["e2e"] = {"value": round(eb / (ems * 1e-3) / 1e9, 1), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                       "ms_per_step": round(ems / K, 4)}
     if rank == 0:
@@ -329,13 +365,121 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def host_link_gbps(torch, gib=1):
+    """Pinned-memory cudaMemcpy bandwidth of this machine, both directions (GB/s), best of 3."""
+    n = gib << 30
+    h = torch.empty(n, dtype=torch.uint8).pin_memory()
+    d = torch.empty(n, dtype=torch.uint8, device="cuda")
+    out = {}
+    for name, (dst, src) in {"h2d": (d, h), "d2h": (h, d)}.items():
+        best = 0.0
+        for _ in range(3):
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(); dst.copy_(src, non_blocking=True); b.record(); torch.cuda.synchronize()
+            best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+        out[name] = round(best, 1)
+    return out
+
+
+def run_lookup(args):
+    """configs[2]: lookup-only stress.  A step is one ptstore_lookup call over 16,384 requests x 64 blocks against a
+    10^6-node trie at load factor 0.7; K steps run back to back between two events."""
+    import torch
+    torch.cuda.set_device(0)
+    from __graft_entry__ import build
+    build()
+    from paper_2607_22648_b200 import binding as G
+    ws = W.lookup_stress()
+    wa = W.lookup_stress(all_hit=True)
+    sh = W.KVShape(1, 1, 8, 16)
+    st = G.PTStore(sh.layers, sh.heads, sh.dim, sh.block_tokens, ws.n_nodes, max_requests=16384, max_batch_blocks=16384 * 64,
+                   table_slots=ws.table_slots, flags=G.lookup_lanes(args.lanes))
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    for i in range(0, len(ws.store_seqs), 8192):
+        t, o = W.ragged(ws.store_seqs[i:i + 8192])
+        st.insert(dev(t), dev(o), 16)
+    assert st.status() == 0
+    res = {}
+    matched = torch.empty(16384, dtype=torch.int32, device="cuda")
+    ids = torch.empty((16384, 64), dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    K, W_ = args.steps, args.warmup
+    sampler = ClockSampler(0)
+    for name, wl, flags in (("geometric_hit_depth", ws, 0), ("geometric_no_touch", ws, G.NO_TOUCH), ("geometric_pin", ws, G.PIN),
+                            ("all_hit", wa, G.NO_TOUCH)):
+        t, o = W.ragged(wl.queries)
+        mb = W.max_blocks_of(wl.queries, 16)
+        dt, do = dev(t), dev(o)
+        m2, i2 = (matched, ids) if mb == 64 else (matched, torch.empty((16384, mb), dtype=torch.int32, device="cuda"))
+        # the timed loop calls the C entry point directly with pre-marshalled arguments: a lookup takes tens of
+        # microseconds, so per-call Python work (tensor attribute lookups, stream object creation) would be measured otherwise
+        stream = torch.cuda.current_stream().cuda_stream
+        cargs = (st.h, dt.data_ptr(), do.data_ptr(), 16384, mb, flags, m2.data_ptr(), i2.data_ptr(), stream)
+        call = G.lib.ptstore_lookup
+        for _ in range(W_):
+            call(*cargs)
+        s0 = st.stats()
+        l0 = st.launch_count()
+        if name == "geometric_hit_depth":
+            sampler.start()
+        # (a) back to back, table and tokens warm in L2
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        t0 = time.perf_counter()
+        for _ in range(K):
+            call(*cargs)
+        host_us = (time.perf_counter() - t0) / K * 1e6
+        b.record(); torch.cuda.synchronize()
+        warm_ms = a.elapsed_time(b) / K
+        if name == "geometric_hit_depth":
+            clocks = sampler.stop()
+        s1 = st.stats()
+        launches = st.launch_count() - l0
+        # (b) L2 flushed before every call
+        cold = []
+        for _ in range(min(K, 10)):
+            flush.fill_(1)
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(); call(*cargs); b.record(); torch.cuda.synchronize()
+            cold.append(a.elapsed_time(b))
+        if flags & G.PIN:
+            for _ in range(W_ + K + len(cold)):
+                st.release(i2, m2)
+        q = (s1.query_blocks - s0.query_blocks) / K
+        pr = (s1.probes_issued - s0.probes_issued) / K
+        res[name] = {"ms_warm": round(warm_ms, 5), "ms_l2_flushed": round(float(np.median(cold)), 5),
+                     "query_blocks_per_s": round(q / (warm_ms * 1e-3)), "issued_probes_per_s": round(pr / (warm_ms * 1e-3)),
+                     "matched_blocks_per_s": round((s1.blocks_matched - s0.blocks_matched) / K / (warm_ms * 1e-3)),
+                     "issued_probes": pr, "query_blocks": q, "slots_per_probe": round((s1.slots_visited - s0.slots_visited) / K / max(pr, 1), 3),
+                     "launches": launches, "host_us_per_call": round(host_us, 2)}
+    assert st.status() == 0
+    main = res["geometric_hit_depth"]
+    peak, kind = measured_peak()
+    # algorithmic bytes of one call: tokens of the hashed blocks (64 B each), one 32-byte sector per probe, 4 B id per query block
+    alg = main["issued_probes"] * (64 + 32) + main["query_blocks"] * 4 + 16384 * 12
+    out = {"metric": "lookup probes/s", "value": main["query_blocks_per_s"], "unit": "query blocks/s", "n_gpus": 1, "steps": K, "warmup": W_,
+           "ms_per_step": main["ms_warm"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64",
+           "data": "synthetic",
+           "config": {"workload": "lookup_stress_1M_nodes_load0.7_16384x64_geometric0.9", "lanes_per_request": args.lanes or "auto",
+                      "l2": "table (22.9 MB) is L2 resident by design; ms_l2_flushed gives the cold figure"},
+           "variants": res, "gpu_launches": main["launches"], "clocks": clocks,
+           "roofline": {"bound": "hbm", "kernel": "lookup_kernel", "achieved": round(alg / (main["ms_warm"] * 1e-3) / 1e9, 1), "peak": peak,
+                        "unit": "GB/s", "frac": round(alg / (main["ms_warm"] * 1e-3) / 1e9 / peak, 4), "traffic": None,
+                        "note": "latency/issue bound, not bandwidth bound: the figure is context only"}}
+    print(json.dumps(out), flush=True)
+
+
 # ---------------------------------------------------------------------------------------------------------
 def cpu_oracle_sample(args, steps=8, batch=8, pool_blocks=2800):
     """The CPU oracle, as it stands, on a bounded sample of the same stream: the same step on the same KV
     shape with `batch` prompts per step and a pool of `pool_blocks` blocks, real bytes moved with memcpy."""
     from oracle import Oracle, PIN
     sh = W.LLAMA3_8B
-    stream = W.llama8b_stream(n_docs=args.docs)
+    stream = W.llama8b_stream(n_docs=args.docs or 500)
     o = Oracle(sh.layers, sh.heads, sh.dim, sh.elem_bytes, sh.block_tokens, 0, pool_blocks, 0, byte_mode=True)
     mb = stream.max_blocks
     B = sh.block_tokens
@@ -379,7 +523,7 @@ def run_reference(args):
     out = {"impl": "reference", "metric": "prefix-hit KV fetch GB/s", "value": res["value"], "unit": "GB/s",
            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W_, "ms_per_step": res["ms_per_step"],
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-           "config": {"workload": Llama8BServing.name, "note": "CPU oracle on a bounded sample of the workload"},
+           "config": {"workload": "llama3_8b_kv_pool20k_zipf1.1_batch64", "note": "CPU oracle on a bounded sample of the workload"},
            "cpu_baseline": res, "e2e": {"value": res["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)
 
@@ -394,9 +538,12 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--fill", type=int, default=6, help="untimed steps that fill the pool before warm-up")
-    ap.add_argument("--batch", type=int, default=64)
-    ap.add_argument("--docs", type=int, default=500)
-    ap.add_argument("--pool-blocks", type=int, default=20000)
+    ap.add_argument("--workload", default="llama8b", choices=["llama8b", "llama70b", "churn", "lookup"])
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--docs", type=int, default=0)
+    ap.add_argument("--pool-blocks", type=int, default=0)
+    ap.add_argument("--host-gb", type=float, default=0.0)
+    ap.add_argument("--lanes", type=int, default=0, help="lookup workload: lanes per request (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per fetch launch, if known (see profiles/)")
@@ -405,6 +552,8 @@ def main():
         args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "lookup":
+        run_lookup(args)
     else:
         run_gpu(args)
 

@@ -246,7 +246,7 @@ int ptstore_last_cuda_error(const ptstore_t* st);
  */
 #define PTSTORE_STATIC_MAX_REQUESTS   1024u
 #define PTSTORE_STATIC_MAX_PAIRS      65536u
-#define PTSTORE_STATIC_SCRATCH_BYTES  (1024u + 4352u + 8u * PTSTORE_STATIC_MAX_PAIRS)
+#define PTSTORE_STATIC_SCRATCH_BYTES  (4096u + 4352u + 8u * PTSTORE_STATIC_MAX_PAIRS)
 int ptstore_fetch_static(const void* hbm_pool, uint32_t hbm_blocks, uint32_t num_layers, uint64_t chunk_bytes,
                          const int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
                          const ptstore_paged_cache_t* dst /*host struct*/, const int32_t* block_tables,

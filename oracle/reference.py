@@ -19,11 +19,16 @@ _lib = None
 
 
 def build_oracle(force=False):
-    """Compile the oracle with g++ if the shared object is missing or older than its source."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    """Compile the oracle with g++ unless the shared object was already built from exactly this source."""
+    import hashlib
+    want = hashlib.sha256(open(_SRC, "rb").read()).hexdigest()
+    stamp = _LIB + ".srchash"
+    if force or not os.path.exists(_LIB) or not os.path.exists(stamp) or open(stamp).read().strip() != want:
         tmp = _LIB + ".tmp%d" % os.getpid()
         subprocess.check_call(["g++", "-std=c++17", "-O2", "-Wall", "-shared", "-fPIC", "-o", tmp, _SRC])
         os.replace(tmp, _LIB)
+        with open(stamp, "w") as f:
+            f.write(want)
     return _LIB
 
 

@@ -11,23 +11,31 @@ NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,c
               "-shared", "-cudart", "shared"]
 
 
-def _newest_source():
-    t = 0.0
+def _source_hash():
+    """Hash of every source and header the library is built from (file times do not survive a copy of the tree)."""
+    import hashlib
+    h = hashlib.sha256()
     for root in (CSRC, os.path.join(os.path.dirname(HERE), "include")):
-        for f in os.listdir(root):
-            t = max(t, os.path.getmtime(os.path.join(root, f)))
-    return t
+        for f in sorted(os.listdir(root)):
+            h.update(f.encode())
+            h.update(open(os.path.join(root, f), "rb").read())
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()
 
 
 def build(force=False, verbose=False):
-    """Compile csrc/*.cu into libptstore.so if it is missing or older than any source."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source():
+    """Compile csrc/*.cu into libptstore.so unless it was already built from exactly these sources."""
+    stamp = LIB + ".srchash"
+    want = _source_hash()
+    if not force and os.path.exists(LIB) and os.path.exists(stamp) and open(stamp).read().strip() == want:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB + ".tmp"] + \
           [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
     os.replace(LIB + ".tmp", LIB)
+    with open(stamp, "w") as f:
+        f.write(want)
     return LIB
 
 

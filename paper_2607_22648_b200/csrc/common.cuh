@@ -29,6 +29,7 @@ constexpr u32 S_NOSPACE = 1u, S_TABLE_FULL = 2u, S_BOUNDS = 4u, S_STATE = 8u, S_
 constexpr u32 F_PIN = 1u, F_NO_TOUCH = 2u;
 
 // ---- control block in device memory ----------------------------------------------------------------
+constexpr int LOOKUP_STRIPES = 64;
 struct Ring {
   u32 head;     // position of the next id to hand out
   u32 count;    // ids available
@@ -50,12 +51,15 @@ struct Ctrl {
   u32 tombstones;
   u32 pad1;
   // cumulative counters
-  u64 query_blocks, probes_issued, slots_visited, blocks_matched;
+  u64 query_blocks, probes_issued, slots_visited, blocks_matched;   // totals are these plus the stripes below
   u64 blocks_fetched[2];
   u64 blocks_inserted, blocks_denied;
   u64 blocks_dropped[2];
   u64 blocks_demoted;
   u64 rebuilds;
+  // lookup counters are striped so that thousands of warps do not queue on four addresses;
+  // [stripe][0..3] = query blocks, probes issued, slots visited, blocks matched
+  u64 lookup_stripes[LOOKUP_STRIPES][4];
 };
 
 // ---- everything a kernel needs to know about the store ---------------------------------------------
@@ -127,16 +131,32 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
   return s;
 }
 
-// Linear probe for `key`.  Returns the slot index or NO_SLOT; *visited gets the slots read.
+// Linear probe for `key`.  Returns the slot index or NO_SLOT; *visited gets the slots examined.
+// The walk is latency bound (each slot is a dependent L2 access) and a warp waits for its slowest lane, so
+// PROBE_WINDOW consecutive slots are loaded at once and then examined in order: a miss at load factor 0.7
+// needs ~6 slots on average with a long tail, which becomes two round trips instead of six or more.
+constexpr int PROBE_WINDOW = 4;
 __device__ __forceinline__ u32 find_slot(const Slot* __restrict__ table, u64 slots, u64 key, u32* visited, u32* id_out) {
   u64 s = home_slot(key, slots);
   u32 n = 0;
-  for (u64 i = 0; i < slots; ++i) {
-    Slot v = load_slot(table + s);
-    ++n;
-    if (v.key == key) { *visited = n; *id_out = v.id; return (u32)s; }
-    if (v.key == KEY_EMPTY) break;
-    s = (s + 1 == slots) ? 0 : s + 1;
+  for (u64 i = 0; i < slots; i += PROBE_WINDOW) {
+    uint4 v[PROBE_WINDOW];
+    u64 idx[PROBE_WINDOW];
+#pragma unroll
+    for (int w = 0; w < PROBE_WINDOW; ++w) {
+      u64 t = s + w;
+      idx[w] = t >= slots ? t - slots : t;
+      v[w] = *reinterpret_cast<const uint4*>(table + idx[w]);
+    }
+#pragma unroll
+    for (int w = 0; w < PROBE_WINDOW; ++w) {
+      const u64 k = ((u64)v[w].y << 32) | v[w].x;
+      ++n;
+      if (k == key) { *visited = n; *id_out = v[w].z; return (u32)idx[w]; }
+      if (k == KEY_EMPTY) { *visited = n; *id_out = NO_ID; return NO_SLOT; }
+    }
+    s += PROBE_WINDOW;
+    if (s >= slots) s -= slots;
   }
   *visited = n;
   *id_out = NO_ID;

@@ -29,7 +29,7 @@ using namespace pts;
 namespace {
 
 constexpr u64 SCR_CTRL = 0;                                                    // Ctrl block
-constexpr u64 SCR_PREFIX = 1024;                                               // u32 [MAX_REQUESTS + 1]
+constexpr u64 SCR_PREFIX = 4096;                                               // u32 [MAX_REQUESTS + 1]
 constexpr u64 SCR_DESC = SCR_PREFIX + ((PTSTORE_STATIC_MAX_REQUESTS + 1) * 4 + 255) / 256 * 256;   // int2 [MAX_PAIRS]
 constexpr u64 SCR_BYTES = SCR_DESC + (u64)PTSTORE_STATIC_MAX_PAIRS * 8;
 static_assert(sizeof(Ctrl) <= SCR_PREFIX, "control block must fit in front of the prefix array");

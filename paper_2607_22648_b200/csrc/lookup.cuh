@@ -60,10 +60,6 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
                                                      int* __restrict__ ids_out) {
   constexpr int G = 32 / L;
   constexpr unsigned SUBMASK = (L == 32) ? FULL : ((1u << L) - 1u);
-  __shared__ u64 s_cnt[4];   // query blocks, probes, slots visited, matched
-  if (threadIdx.x < 4) s_cnt[threadIdx.x] = 0;
-  __syncthreads();
-
   const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long r = warp * G + sub;
@@ -124,24 +120,15 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
     for (int j = m + sl; j < max_blocks; j += L) ids_out[r * max_blocks + j] = -1;
     if (sl == 0) matched[r] = m;
   }
-  // counters: warp sums, then one atomic per block and counter
+  // counters: warp sums, then fire-and-forget adds into one of LOOKUP_STRIPES stripes (no block barrier)
   u32 qb = (valid && sl == 0) ? (u32)nblk : 0, mb = (valid && sl == 0) ? (u32)m : 0;
   qb = __reduce_add_sync(FULL, qb);
   mb = __reduce_add_sync(FULL, mb);
   my_probes = __reduce_add_sync(FULL, my_probes);
   my_visited = __reduce_add_sync(FULL, my_visited);
-  if (lane == 0) {
-    atomicAdd(&s_cnt[0], (u64)qb);
-    atomicAdd(&s_cnt[1], (u64)my_probes);
-    atomicAdd(&s_cnt[2], (u64)my_visited);
-    atomicAdd(&s_cnt[3], (u64)mb);
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    if (s_cnt[0]) atomicAdd(&st.ctrl->query_blocks, s_cnt[0]);
-    if (s_cnt[1]) atomicAdd(&st.ctrl->probes_issued, s_cnt[1]);
-    if (s_cnt[2]) atomicAdd(&st.ctrl->slots_visited, s_cnt[2]);
-    if (s_cnt[3]) atomicAdd(&st.ctrl->blocks_matched, s_cnt[3]);
+  if (lane < 4) {
+    const u32 v = lane == 0 ? qb : lane == 1 ? my_probes : lane == 2 ? my_visited : mb;
+    if (v) atomicAdd(&st.ctrl->lookup_stripes[warp % LOOKUP_STRIPES][lane], (u64)v);
   }
 }
 
