@@ -230,6 +230,23 @@ class Serving:
         return h2d, d2h
 
 
+def reduce_over_ranks(dist, x, op, device):
+    """max or sum of a python number over all ranks (identity without a process group)."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def whole_job_throughput(dist, ms, nbytes, device):
+    """Replicas: the job's time is the slowest rank's, its work the sum over ranks.  -> (ms, bytes, GB/s)"""
+    ms_all = reduce_over_ranks(dist, ms, "max", device)
+    bytes_all = reduce_over_ranks(dist, nbytes, "sum", device)
+    return ms_all, bytes_all, bytes_all / (ms_all * 1e-3) / 1e9
+
+
 def run_gpu(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -307,19 +324,10 @@ def run_gpu(args):
 
     # aggregate over ranks: max time, sum of bytes
     def agg(x, op):
-        if not dist:
-            return x
-        t = torch.tensor([float(x)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=op)
-        return float(t.item())
+        return reduce_over_ranks(dist, x, op, "cuda")
 
-    if dist:
-        MAX, SUM = dist.ReduceOp.MAX, dist.ReduceOp.SUM
-    else:
-        MAX = SUM = None
-    ms = agg(main["ms"], MAX)
-    total_bytes = agg(main["bytes"], SUM)
-    value = total_bytes / (ms * 1e-3) / 1e9
+    MAX, SUM = "max", "sum"
+    ms, total_bytes, value = whole_job_throughput(dist, main["ms"], main["bytes"], "cuda")
     peak, peak_kind = measured_peak()
     fetch_bytes = main["fetched"] * block_rw
     ach = fetch_bytes / (fetch_ms * 1e-3) / 1e9 if fetch_ms > 0 else 0.0
