@@ -131,11 +131,10 @@ class Serving:
             self.name = "llama3_70b_kv_pool%d_zipf1.2_batch%d_16k_prefix" % (self.pool_blocks, self.batch)
             self.kv = "80L x 8H x 128 bf16, block 32"
         else:
-            import psutil
             self.sh = W.LLAMA3_8B
             self.batch, self.pool_blocks = args.batch or 16, args.pool_blocks or 19073
             self.stream = W.churn_stream(seed=W.BASE_SEED + 4 + 1000 * rank, n_docs=args.docs or 5000)
-            host_gb = args.host_gb if args.host_gb else min(200.0, psutil.virtual_memory().available / 1e9 * 0.4)
+            host_gb = args.host_gb if args.host_gb else pinnable_host_gb()
             host_blocks = int(host_gb * 1e9 // self.sh.block_bytes)
             self.name = "churn_llama3_8b_kv_hbm%d_host%d_zipf1.0_batch%d" % (self.pool_blocks, host_blocks, self.batch)
             self.kv = "32L x 8H x 128 bf16, block 16"
@@ -371,6 +370,20 @@ def run_gpu(args):
     if dist:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def pinnable_host_gb(fraction=0.4, cap=200.0):
+    """Budget for the pinned host pool: a fraction of the available RAM, never above the cgroup limit."""
+    import psutil
+    avail = psutil.virtual_memory().available / 1e9
+    for path in ("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory/memory.limit_in_bytes"):
+        try:
+            lim = open(path).read().strip()
+            if lim != "max":
+                avail = min(avail, int(lim) / 1e9)
+        except Exception:
+            pass
+    return max(1.0, min(cap, avail * fraction))
 
 
 def host_link_gbps(torch, gib=1):

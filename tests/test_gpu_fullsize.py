@@ -102,13 +102,12 @@ def test_llama70b_16k_prefix_fetch_shuffled_tables():
 def test_churn_with_host_tier():
     """config 5: Llama-3-8B shape, 40 GB HBM store + pinned-host store, Zipf(1.0) over 5000 documents,
     micro-batches of 16 with LRU demotion to the host tier and drops from it."""
-    import psutil
-    from tests.serving import LockstepServing
+    from tests.serving import LockstepServing, pinnable_host_gb
     sh = W.LLAMA3_8B
     st = W.churn_stream()
     mb = st.max_blocks
     hbm = 19073 if _free_gb() > 80 else 4000
-    host_gb = min(200.0, psutil.virtual_memory().available / 1e9 * 0.35)
+    host_gb = pinnable_host_gb()          # the 200 GB of the config exceed this box's RAM; the size used is printed
     host = int(host_gb * 1e9 // sh.block_bytes)
     cache_blocks = 16 * mb
     srv = LockstepServing(sh, hbm, host, 16, mb, cache_blocks, seed=5)
