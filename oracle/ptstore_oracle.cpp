@@ -394,6 +394,45 @@ void oracle_evict(void* h, int32_t tier, int32_t n, int32_t mode, int32_t* n_evi
   n_evicted[1] = nd;
 }
 
+// Promotion of host-tier blocks named by a batch into HBM (the paper keeps hot prefixes on the fastest tier,
+// Section 4.1 "Replication of popular prefixes"; with one store the analogue is moving a hit block from the
+// host pool to the HBM pool).  Reading: entries are visited in (request, block) order, so the front of a
+// prefix goes first; a block moves only if nobody outside this list holds its id (refcount equals the
+// list's own pins, or 0 for an unpinned list), while the budget lasts and the HBM free list is not empty.
+// Every entry naming a moved block is rewritten to the new id.
+void oracle_promote(void* h, int32_t* ids, const int32_t* matched, int32_t R, int32_t maxB, uint32_t pinned_list,
+                    int32_t max_promote, int32_t* n_promoted) {
+  Oracle* o = (Oracle*)h;
+  int32_t total = o->n[0] + o->n[1];
+  std::map<int32_t, int64_t> count;                 // how many entries of this list name each block
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < matched[r] && j < maxB; ++j) count[ids[(int64_t)r * maxB + j]] += 1;
+  std::map<int32_t, int32_t> moved;
+  int P = 0;
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < matched[r] && j < maxB; ++j) {
+      int32_t& id = ids[(int64_t)r * maxB + j];
+      auto mv = moved.find(id);
+      if (mv != moved.end()) { id = mv->second; continue; }              // moved earlier in this call: rewrite
+      if (id < o->n[0] || id >= total || !o->by_id[id]) continue;       // HBM already, or not a live block
+      if (P >= max_promote || o->free_list[TIER_HBM].empty()) continue;
+      Node* nd = o->by_id[id];
+      if (nd->refcount != (pinned_list ? count[id] : 0)) continue;
+      int32_t new_id = o->free_list[TIER_HBM].front();
+      o->free_list[TIER_HBM].pop_front();
+      if (o->byte_mode) std::memcpy(o->block_ptr(new_id), o->block_ptr(id), o->block_bytes);
+      o->by_id[id] = nullptr;
+      o->by_id[new_id] = nd;
+      nd->block_id = new_id;
+      nd->tier = TIER_HBM;
+      o->free_list[TIER_HOST].push_back(id);
+      moved[id] = new_id;
+      id = new_id;
+      ++P;
+    }
+  *n_promoted = P;
+}
+
 uint32_t oracle_status(void* h) { Oracle* o = (Oracle*)h; uint32_t s = o->status; o->status = 0; return s; }
 uint64_t oracle_epoch(void* h) { return ((Oracle*)h)->epoch; }
 uint64_t oracle_collisions(void* h) { return ((Oracle*)h)->collisions; }

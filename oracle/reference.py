@@ -50,6 +50,7 @@ def _load():
         lib.oracle_insert.argtypes = [vp, vp, vp, i32, i32, vp, u64, u64, C.c_uint32, vp, vp, vp, vp]
         lib.oracle_release.argtypes = [vp, vp, vp, i32, i32]
         lib.oracle_evict.argtypes = [vp, i32, i32, i32, vp, vp]
+        lib.oracle_promote.argtypes = [vp, vp, vp, i32, i32, C.c_uint32, i32, vp]
         lib.oracle_status.restype = C.c_uint32; lib.oracle_status.argtypes = [vp]
         lib.oracle_epoch.restype = u64; lib.oracle_epoch.argtypes = [vp]
         lib.oracle_collisions.restype = u64; lib.oracle_collisions.argtypes = [vp]
@@ -165,6 +166,14 @@ class Oracle:
         victims = np.full(max(2 * n, 1), -1, dtype=np.int32)
         self.lib.oracle_evict(self.h, tier, n, 0 if literal else 1, _p(ne), _p(victims))
         return ne, victims[: int(ne[0] + ne[1])]
+
+    def promote(self, ids, matched, pinned_list, max_promote):
+        """Moves host-tier blocks of the list into HBM; returns (rewritten ids, number moved)."""
+        ids, matched = _i32(ids).copy(), _i32(matched)
+        R, maxB = ids.shape
+        n = np.zeros(1, dtype=np.int32)
+        self.lib.oracle_promote(self.h, _p(ids), _p(matched), R, maxB, 1 if pinned_list else 0, int(max_promote), _p(n))
+        return ids, int(n[0])
 
     # -- introspection -------------------------------------------------------------------------------
     def status(self):

@@ -490,3 +490,68 @@ def test_demote_makes_room_by_dropping_host_first():
     assert m.tolist() == [0, 0, 1, 1, 1, 1]
     assert ids[:, 0].tolist() == [-1, -1, 8, 6, 7, 5]
     check_invariants(o)
+
+
+# ---- promotion of host-tier blocks ----------------------------------------------------------------------------
+def test_promotion_front_of_prefix_first_with_budget_and_pins():
+    sh = W.KVShape(2, 1, 8, 2)
+    B = 2
+    o = Oracle(sh.layers, sh.heads, sh.dim, 2, B, 0, 8, 6)
+    rng = np.random.default_rng(0)
+    a = np.array([1, 1, 2, 2, 3, 3, 4, 4], dtype=np.int32)
+    b = np.array([1, 1, 5, 5], dtype=np.int32)
+    src = W.random_kv_cache(1, sh, 8)
+    bt = W.shuffled_block_tables(rng, [a, b], B, 4, 8)
+    o.insert(*W.ragged([a, b]), 4, src, bt)                                 # ids a: 0 1 2 3, b: 0 4
+    original = {i: o.pool(0)[i].copy() for i in range(5)}
+    ne, v = o.evict(0, 5)                                                   # everything goes to host, deepest first
+    assert ne.tolist() == [5, 0] and v.tolist() == [3, 2, 1, 4, 0]          # host ids 8 9 10 11 12 in that order
+    m, ids = o.lookup(*W.ragged([a, b]), 4, PIN)
+    assert ids.tolist() == [[12, 10, 9, 8], [12, 11, -1, -1]]
+    # budget 3: the shared first block, then a's second and third (front of the prefix first); HBM ids from the ring front
+    new_ids, n = o.promote(ids, m, True, 3)
+    assert n == 3 and new_ids.tolist() == [[5, 6, 7, 8], [5, 11, -1, -1]]
+    assert o.free_list(0).tolist() == [3, 2, 1, 4, 0] and o.free_list(1).tolist() == [13, 12, 10, 9]
+    for new, old in ((5, 0), (6, 1), (7, 2)):
+        assert (o.pool(0)[new] == original[old]).all()                      # bytes travelled with the node
+    info = o.block_info(5)
+    assert info["refcount"] == 2 and info["depth"] == 0 and o.block_info(6)["parent"] == 5
+    check_invariants(o)
+    # a second list pinning the same blocks: a block whose count exceeds this list's own pins stays where it is
+    m2, ids2 = o.lookup(*W.ragged([b]), 4, PIN)                              # pins 5 and 11 once more
+    moved, n = o.promote(new_ids, m, True, 10)                               # list 1 names 11 once, its refcount is 2
+    assert n == 1 and moved.tolist() == [[5, 6, 7, 3], [5, 11, -1, -1]]       # only a's last block (8) can move
+    o.release(ids2, m2)
+    o.release(moved, m)
+    assert all(nd["refcount"] == 0 for nd in all_nodes(o).values())
+    # unpinned list: moves only blocks nobody pins
+    m3, ids3 = o.lookup(*W.ragged([b]), 4)
+    moved3, n = o.promote(ids3, m3, False, 10)
+    assert n == 1 and moved3.tolist() == [[5, 2, -1, -1]]
+    check_invariants(o)
+    assert o.live_count(1) == 0 and o.free_count(1) == 6
+    # no free HBM block, or no budget: nothing moves
+    o.evict(0, 2)
+    m4, ids4 = o.lookup(*W.ragged([a]), 4)
+    same, n = o.promote(ids4, m4, False, 0)
+    assert n == 0 and (same == ids4).all()
+
+
+def test_promotion_random_histories_keep_invariants_and_lookup_results():
+    for seed in range(30):
+        o, seqs, mb, rng = random_store(seed + 500, pool=40, host=40)
+        o.evict(0, int(rng.integers(5, 40)), literal=False)
+        for step in range(6):
+            batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(3)]
+            toks, offs = W.ragged(batch)
+            m, ids = o.lookup(toks, offs, mb, PIN)
+            hbm_free = o.free_count(0)
+            host_named = len({int(i) for r in range(len(m)) for i in ids[r, :m[r]] if i >= o.hbm_blocks})
+            budget = int(rng.integers(0, 8))
+            new_ids, n = o.promote(ids, m, True, budget)
+            assert n <= min(budget, hbm_free, host_named)
+            m2, ids2 = o.lookup(toks, offs, mb, NO_TOUCH)                   # same matches, ids as rewritten
+            assert (m2 == m).all() and (ids2 == new_ids).all()
+            o.release(new_ids, m)
+            check_invariants(o)
+            o.evict(0, int(rng.integers(0, 6)), literal=bool(step % 2))
