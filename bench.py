@@ -139,6 +139,7 @@ class Serving:
             self.name = "churn_llama3_8b_kv_hbm%d_host%d_zipf1.0_batch%d" % (self.pool_blocks, host_blocks, self.batch)
             self.kv = "32L x 8H x 128 bf16, block 16"
         self.host_blocks = host_blocks
+        self.promote = args.promote if host_blocks else 0
         self.mb = self.stream.max_blocks
         flags = (G.COPY_BULK if args.engine == "bulk" else G.COPY_VECTOR) | G.copy_variant(args.variant) | \
             G.copy_ctas_per_sm(args.ctas_per_sm)
@@ -178,6 +179,7 @@ class Serving:
         self.ins_ids = torch.empty((R, self.mb), dtype=torch.int32, device="cuda")
         self.newb = torch.empty(R, dtype=torch.int32, device="cuda")
         self.nev = torch.zeros(2, dtype=torch.int32, device="cuda")
+        self.nprom = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.h_matched = torch.empty(R, dtype=torch.int32).pin_memory()
         self.h_ids = torch.empty((R, self.mb), dtype=torch.int32).pin_memory()
         self.h_newb = torch.empty(R, dtype=torch.int32).pin_memory()
@@ -191,6 +193,12 @@ class Serving:
         else:
             d = s["dev"]
         st.lookup(d["tokens"], d["offsets"], self.mb, G.PIN, self.matched, self.ids)
+        if self.promote:
+            if events is not None:
+                events["promote"].append((self._ev(), None))
+            st.promote(self.ids, self.matched, G.PINNED_LIST, self.promote, self.nprom)
+            if events is not None:
+                events["promote"][-1] = (events["promote"][-1][0], self._ev())
         if events is not None:
             events["fetch"].append((self._ev(), None))
         st.fetch(self.ids, self.matched, self.cache, d["bt"])
@@ -199,7 +207,7 @@ class Serving:
         # the serving engine needs the matched lengths on the host anyway; the same sync gives the free count
         self.h_matched.copy_(self.matched, non_blocking=True)
         stats = st.stats()
-        need = s["total_blocks"] - int(self.h_matched.sum())
+        need = s["total_blocks"] - int(self.h_matched.sum()) + self.promote      # keep room for the next step's promotions
         short = need - int(stats.free_blocks[0])
         if short > 0:
             if events is not None:
@@ -289,10 +297,11 @@ def run_gpu(args):
         ms = t0.elapsed_time(t1)
         s1 = wl.store.stats()
         fetched = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) + (s1.blocks_fetched[1] - s0.blocks_fetched[1])
-        moved = fetched + (s1.blocks_inserted - s0.blocks_inserted) + (s1.blocks_demoted - s0.blocks_demoted)
+        moved = fetched + (s1.blocks_inserted - s0.blocks_inserted) + (s1.blocks_demoted - s0.blocks_demoted) + \
+            (s1.blocks_promoted - s0.blocks_promoted)
         return dict(ms=ms, fetched=fetched, fetched_host=s1.blocks_fetched[1] - s0.blocks_fetched[1],
                     inserted=s1.blocks_inserted - s0.blocks_inserted, demoted=s1.blocks_demoted - s0.blocks_demoted,
-                    host_dropped=s1.blocks_dropped[1] - s0.blocks_dropped[1],
+                    host_dropped=s1.blocks_dropped[1] - s0.blocks_dropped[1], promoted=s1.blocks_promoted - s0.blocks_promoted,
                     bytes=moved * block_rw, launches=wl.store.launch_count() - l0,
                     probes=s1.probes_issued - s0.probes_issued, qblocks=s1.query_blocks - s0.query_blocks,
                     matched=s1.blocks_matched - s0.blocks_matched, dropped=s1.blocks_dropped[0] - s0.blocks_dropped[0])
@@ -303,7 +312,7 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    events = {"fetch": [], "insert": [], "evict": []}
+    events = {"fetch": [], "insert": [], "evict": [], "promote": []}
     main = timed(i, K, False, events)
     clocks = sampler.stop() if rank == 0 else None
     i += K
@@ -311,6 +320,7 @@ def run_gpu(args):
     fetch_ms = sum(a.elapsed_time(b) for a, b in events["fetch"])
     insert_ms = sum(a.elapsed_time(b) for a, b in events["insert"])
     evict_ms = sum(a.elapsed_time(b) for a, b in events["evict"])
+    promote_ms = sum(a.elapsed_time(b) for a, b in events["promote"])
     status = wl.store.status()
 
     e2e = None
@@ -344,7 +354,8 @@ def run_gpu(args):
                      "insert_gbps": round(main["inserted"] * block_rw / max(insert_ms, 1e-9) / 1e6, 1),
                      "lookup_probes": main["probes"] / K, "blocks_fetched_from_host": main["fetched_host"] / K,
                      "blocks_demoted": main["demoted"] / K, "host_blocks_dropped": main["host_dropped"] / K,
-                     "evict_call_ms": round(evict_ms / K, 4),
+                     "evict_call_ms": round(evict_ms / K, 4), "blocks_promoted": main["promoted"] / K,
+                     "promote_call_ms": round(promote_ms / K, 4),
                      "demote_gbps_one_way": round(main["demoted"] * wl.sh.block_bytes / max(evict_ms, 1e-9) / 1e6, 1)},
         "gpu_launches": int(main["launches"]),
         "device_status": status,
@@ -564,6 +575,7 @@ def main():
     ap.add_argument("--docs", type=int, default=0)
     ap.add_argument("--pool-blocks", type=int, default=0)
     ap.add_argument("--host-gb", type=float, default=0.0)
+    ap.add_argument("--promote", type=int, default=0, help="churn workload: host-tier blocks promoted into HBM per step (budget)")
     ap.add_argument("--lanes", type=int, default=0, help="lookup workload: lanes per request (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -62,6 +62,9 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 #define PTSTORE_PIN       0x1u   /* refcount++ on every matched (request, block) pair */
 #define PTSTORE_NO_TOUCH  0x2u   /* do not refresh the LRU stamp of matched blocks */
 
+/* flags of ptstore_promote */
+#define PTSTORE_PINNED_LIST 0x1u  /* the id list passed in was produced by a lookup with PTSTORE_PIN */
+
 /* flags of ptstore_config_t */
 #define PTSTORE_COPY_VECTOR  0x0u  /* copy engine: 16-byte vector loads/stores (always used for the host tier) */
 #define PTSTORE_COPY_BULK    0x1u  /* copy engine: bulk-async copies through a shared-memory ring (HBM<->HBM) */
@@ -117,6 +120,7 @@ typedef struct {                 /* all counters are cumulative since create */
   uint64_t blocks_dropped[2];    /* deleted per tier */
   uint64_t blocks_demoted;       /* HBM -> host */
   uint64_t rebuilds;
+  uint64_t blocks_promoted;      /* host -> HBM */
 } ptstore_stats_t;
 
 /*
@@ -215,6 +219,23 @@ int ptstore_release(ptstore_t* st, const int32_t* block_ids, const int32_t* matc
  */
 int ptstore_evict(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids,
                   ptstore_stream_t stream);
+
+/*
+ * Move host-tier blocks named by a batch into HBM (the paper keeps hot prefixes on the fastest tier, Section 4.1
+ * "Replication of popular prefixes to improve access locality"; with one store the analogue is promoting a block
+ * that was just hit).  Entries (r, j < matched_blocks[r]) are taken in (r, j) order, so the front of a prefix
+ * moves first.  A block moves at most once per call, and only while (a) fewer than max_promote blocks have moved,
+ * (b) the HBM free ring is not empty, and (c) nobody else holds its id: its reference count equals the number of
+ * entries of this list that name it (flags = PTSTORE_PINNED_LIST) or zero (flags = 0).  The block gets the id at
+ * the front of the HBM ring, its bytes are copied host -> HBM, its node keeps its place and stamps, and the host
+ * id goes to the back of the host ring.
+ *   block_ids   in/out [R*max_blocks]: entries naming a moved block are rewritten to its new id (use the
+ *               rewritten list for the following fetch and release)
+ *   n_promoted  out, device [1] or NULL: blocks moved
+ * No host tier: returns PTSTORE_E_INVAL.  Call it between lookup and fetch.
+ */
+int ptstore_promote(ptstore_t* st, int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
+                    uint32_t flags, int32_t max_promote, int32_t* n_promoted, ptstore_stream_t stream);
 
 /* Synchronise `stream`, read the device status word into *status_out (host) and clear it. */
 int ptstore_status(ptstore_t* st, ptstore_stream_t stream, uint32_t* status_out /*host*/);

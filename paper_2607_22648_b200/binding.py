@@ -13,6 +13,7 @@ from . import build as _build
 OK, E_INVAL, E_CUDA, E_NOMEM, E_LIMIT = 0, -1, -2, -3, -4
 S_NOSPACE, S_TABLE_FULL, S_BOUNDS, S_STATE, S_TIMEOUT = 1, 2, 4, 8, 16
 PIN, NO_TOUCH = 1, 2
+PINNED_LIST = 1
 COPY_VECTOR, COPY_BULK = 0, 1
 TIER_HBM, TIER_HOST = 0, 1
 
@@ -50,12 +51,12 @@ class Stats(C.Structure):
                 ("tombstones", C.c_uint64), ("query_blocks", C.c_uint64), ("probes_issued", C.c_uint64),
                 ("slots_visited", C.c_uint64), ("blocks_matched", C.c_uint64), ("blocks_fetched", C.c_uint64 * 2),
                 ("blocks_inserted", C.c_uint64), ("blocks_denied", C.c_uint64), ("blocks_dropped", C.c_uint64 * 2),
-                ("blocks_demoted", C.c_uint64), ("rebuilds", C.c_uint64)]
+                ("blocks_demoted", C.c_uint64), ("rebuilds", C.c_uint64), ("blocks_promoted", C.c_uint64)]
 
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
-           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static"]
+           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote"]
 
 
 def _load():
@@ -74,6 +75,7 @@ def _load():
     lib.ptstore_insert.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
     lib.ptstore_release.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.ptstore_evict.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.ptstore_promote.argtypes = [vp, vp, vp, i32, i32, u32, i32, vp, vp]
     lib.ptstore_status.argtypes = [vp, vp, C.POINTER(u32)]
     lib.ptstore_stats.argtypes = [vp, vp, C.POINTER(Stats)]
     lib.ptstore_launch_count.restype = u64
@@ -228,6 +230,15 @@ class PTStore:
             victims = torch.full((max(2 * n, 1),), -1, dtype=torch.int32, device=self.device)
         self._check(lib.ptstore_evict(self.h, tier, n, _ptr(n_evicted), _ptr(victims), _stream()), "ptstore_evict")
         return n_evicted, victims
+
+    def promote(self, ids, matched, flags, max_promote, n_promoted=None):
+        """Rewrites `ids` in place; returns the device counter of blocks moved."""
+        R, mb = ids.shape
+        if n_promoted is None:
+            n_promoted = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self._check(lib.ptstore_promote(self.h, _ptr(ids), _ptr(matched), R, mb, flags, max_promote, _ptr(n_promoted), _stream()),
+                    "ptstore_promote")
+        return n_promoted
 
     def status(self):
         out = C.c_uint32(0)

@@ -57,6 +57,7 @@ struct Ctrl {
   u64 blocks_dropped[2];
   u64 blocks_demoted;
   u64 rebuilds;
+  u64 blocks_promoted;
   // lookup counters are striped so that thousands of warps do not queue on four addresses;
   // [stripe][0..3] = query blocks, probes issued, slots visited, blocks matched
   u64 lookup_stripes[LOOKUP_STRIPES][4];

@@ -12,6 +12,7 @@
 #include "copy.cuh"
 #include "insert.cuh"
 #include "evict.cuh"
+#include "promote.cuh"
 
 using namespace pts;
 
@@ -22,7 +23,7 @@ inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
   u64 table[2], m_key, m_parent, m_last, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
-      cta_sums, prefix, total;
+      cta_sums, prefix, promo_first, promo_cnt, total;
   u32 n_tiles;
 };
 
@@ -59,6 +60,8 @@ Layout make_layout(const ptstore_config_t* c) {
   L.eslot = take(M * 4);
   L.cta_sums = take(((M + INS_THREADS - 1) / INS_THREADS + 1) * 4);
   L.prefix = take(((u64)c->max_requests + 1) * 4);
+  L.promo_first = take(N * 4);
+  L.promo_cnt = take(N * 4);
   L.total = o;
   return L;
 }
@@ -81,6 +84,8 @@ struct ptstore {
   u32* eslot;
   u32* cta_sums;
   u32* prefix;
+  u32* promo_first;
+  u32* promo_cnt;
   u64 epoch;
   u64 launches;
   int last_cuda;
@@ -379,6 +384,8 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->eslot = reinterpret_cast<u32*>(w + lay.eslot);
   h->cta_sums = reinterpret_cast<u32*>(w + lay.cta_sums);
   h->prefix = reinterpret_cast<u32*>(w + lay.prefix);
+  h->promo_first = reinterpret_cast<u32*>(w + lay.promo_first);
+  h->promo_cnt = reinterpret_cast<u32*>(w + lay.promo_cnt);
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int cap = sms * 8;
@@ -529,6 +536,41 @@ int ptstore_evict(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evict
   return launch_copy<COPY_POOL>(h, none, true, s);
 }
 
+int ptstore_promote(ptstore_t* h, int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks, uint32_t flags,
+                    int32_t max_promote, int32_t* n_promoted, ptstore_stream_t stream) {
+  int rc = check_batch(h, R, max_blocks);
+  if (rc) return rc;
+  if (h->cfg.host_blocks == 0 || max_promote < 0) return PTSTORE_E_INVAL;
+  if (R > 0 && (!block_ids || !matched_blocks)) return PTSTORE_E_INVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
+  if (cudaMemsetAsync(h->promo_first, 0xFF, N * 4, s) != cudaSuccess || cudaMemsetAsync(h->promo_cnt, 0, N * 4, s) != cudaSuccess) {
+    h->last_cuda = (int)cudaGetLastError();
+    return PTSTORE_E_CUDA;
+  }
+  const long long total = (long long)R * max_blocks;
+  const int cap = h->sms * 8;
+  const u32 pinned = (flags & PTSTORE_PINNED_LIST) ? 1u : 0u;
+  const u32 n_ctas = (u32)((total + INS_THREADS - 1) / INS_THREADS);
+  if (total > 0) {
+    promote_mark_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first, h->promo_cnt);
+    PTS_CHECK_LAUNCH(h);
+    promote_count_kernel<<<n_ctas, INS_THREADS, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first, h->promo_cnt,
+                                                        pinned, h->cta_sums);
+    PTS_CHECK_LAUNCH(h);
+  }
+  promote_plan_kernel<<<1, INS_THREADS, 0, s>>>(h->st, h->cta_sums, total > 0 ? n_ctas : 0, (u32)max_promote, n_promoted);
+  PTS_CHECK_LAUNCH(h);
+  if (total == 0) return PTSTORE_OK;
+  promote_assign_kernel<<<n_ctas, INS_THREADS, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first, h->promo_cnt,
+                                                       pinned, h->cta_sums, h->desc);
+  PTS_CHECK_LAUNCH(h);
+  promote_rewrite_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first);
+  PTS_CHECK_LAUNCH(h);
+  Paged none = {};
+  return launch_copy<COPY_POOL>(h, none, true, s);
+}
+
 int ptstore_status(ptstore_t* h, ptstore_stream_t stream, uint32_t* status_out) {
   if (!h || !status_out) return PTSTORE_E_INVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -571,6 +613,7 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
   out->blocks_denied = c.blocks_denied;
   out->blocks_demoted = c.blocks_demoted;
   out->rebuilds = c.rebuilds;
+  out->blocks_promoted = c.blocks_promoted;
   return PTSTORE_OK;
 }
 

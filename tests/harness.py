@@ -70,6 +70,14 @@ class Pair:
         assert (no == ng.cpu().numpy()).all(), "new block counts differ"
         return io, no
 
+    def promote(self, ids, matched, pinned_list, max_promote):
+        new_o, n_o = self.o.promote(ids, matched, pinned_list, max_promote)
+        ig = dev(ids)
+        n_g = self.g.promote(ig, dev(matched), G.PINNED_LIST if pinned_list else 0, max_promote)
+        assert n_o == int(n_g.item()), ("promoted counts differ", n_o, int(n_g.item()))
+        assert (new_o == ig.cpu().numpy()).all(), "rewritten ids differ"
+        return new_o, n_o
+
     def release(self, ids, matched):
         self.o.release(ids, matched)
         self.g.release(dev(ids), dev(matched))

@@ -112,16 +112,18 @@ def test_churn_with_host_tier():
     cache_blocks = 16 * mb
     srv = LockstepServing(sh, hbm, host, 16, mb, cache_blocks, seed=5)
     n_steps = 60
-    demoted = dropped = 0
+    demoted = dropped = promoted = 0
     for k in range(n_steps):
         seqs, tags = st.batch(16)
-        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9))
+        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9), promote=(256 if k >= 30 else 0))
+        promoted += r["promoted"]
         if r["evicted"] is not None:
             demoted += int(r["evicted"][0]); dropped += int(r["evicted"][1])
     s = srv.check_counts()
     assert srv.check_pool(32) > 0
     assert demoted > 0 and s.blocks_demoted == demoted
+    assert promoted > 0 and s.blocks_promoted == promoted
     assert srv.sampled_chunks >= 256
-    print("churn: hbm %d blocks, host %d blocks (%.0f GB pinned), %d steps, demoted %d, host drops %d, fetched from hbm/host %s"
-          % (hbm, host, host * sh.block_bytes / 1e9, n_steps, demoted, dropped, srv.fetched_by_tier))
+    print("churn: hbm %d blocks, host %d blocks (%.0f GB pinned), %d steps, demoted %d, host drops %d, promoted %d, fetched from hbm/host %s"
+          % (hbm, host, host * sh.block_bytes / 1e9, n_steps, demoted, dropped, promoted, srv.fetched_by_tier))
     srv.close()

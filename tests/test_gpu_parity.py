@@ -151,6 +151,8 @@ def test_random_churn_lockstep(host):
             for r in range(len(batch)):
                 for j in range(mo[r]):
                     bt[r, j] = perm[k]; k += 1
+            if host and rng.random() < 0.6:                    # move some of the host-tier hits into HBM first
+                io, _n = p.promote(io, mo, True, int(rng.integers(0, 6)))
             p.fetch(io, mo, dst, bt)
             if op < 0.7:
                 tier = int(rng.integers(0, 2)) if host else 0
@@ -173,6 +175,43 @@ def test_random_churn_lockstep(host):
         p.check_pools()
         s = p.check_counts()
         p.close()
+
+
+def test_promotion_worked_example_and_unpinned_lists():
+    Pair, dev, G = _imports()
+    sh = W.KVShape(2, 1, 8, 2)
+    p = Pair(sh, 8, host_blocks=6, max_requests=4, max_batch_blocks=16)
+    rng = np.random.default_rng(0)
+    a = np.array([1, 1, 2, 2, 3, 3, 4, 4], dtype=np.int32)
+    b = np.array([1, 1, 5, 5], dtype=np.int32)
+    src = W.random_kv_cache(1, sh, 8)
+    p.insert([a, b], 4, src, W.shuffled_block_tables(rng, [a, b], 2, 4, 8))
+    p.evict(0, 5)
+    mo, io, _, _ = p.lookup([a, b], 4, flags=1)
+    new_ids, n = p.promote(io, mo, True, 3)
+    assert n == 3 and new_ids.tolist() == [[5, 6, 7, 8], [5, 11, -1, -1]]
+    p.check_pools()
+    p.check_counts()
+    dst = [np.zeros((2, 8, sh.chunk_bytes), dtype=np.uint8) for _ in range(sh.layers)]
+    p.fetch(new_ids, mo, dst, np.array([[0, 1, 2, 3], [4, 5, -1, -1]], dtype=np.int32))
+    mo2, io2, _, _ = p.lookup([b], 4, flags=1)
+    moved, n = p.promote(new_ids, mo, True, 10)
+    assert n == 1 and moved.tolist() == [[5, 6, 7, 3], [5, 11, -1, -1]]
+    p.release(io2, mo2)
+    p.release(moved, mo)
+    mo3, io3, _, _ = p.lookup([b], 4)
+    moved3, n = p.promote(io3, mo3, False, 10)
+    assert n == 1 and moved3.tolist() == [[5, 2, -1, -1]]
+    same, n = p.promote(moved3, mo3, False, 0)
+    assert n == 0
+    p.lookup([a, b], 4)
+    assert p.check_status() == 0
+    p.check_pools()
+    s = p.check_counts()
+    assert s.blocks_promoted == 5 and s.live_nodes[1] == 0
+    with pytest.raises(G.PTStoreError):
+        Pair(sh, 8).g.promote(dev(io3), dev(mo3), 0, 1)          # no host tier
+    p.close()
 
 
 def test_lookup_stress_small_matches_oracle():
