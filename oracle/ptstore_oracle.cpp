@@ -77,7 +77,8 @@ struct Node {
   int32_t block_id;    // pool block that holds its K/V
   int tier;
   int64_t refcount;
-  u64 last_use;
+  u64 last_use;        // LRU policy: stamp of the last touch.  GDSF policy: the priority H = L + F at the last touch
+  u64 freq;            // GDSF policy: number of accesses F
   u64 key;             // chained key, computed for comparison with the GPU path only
   u64 tag;             // tag mode: identity of the payload
   std::vector<int32_t> tokens;
@@ -100,6 +101,8 @@ struct Oracle {
   std::map<u64, Node*> by_key;        // only to DETECT two token paths with one key
   u64 collisions;
   u64 epoch;
+  int policy;                         // 0 = LRU, 1 = GDSF with equal size and cost per block
+  u64 inflation;                      // GDSF clock L: the largest priority evicted so far
   uint32_t status;
   Node root;
 
@@ -123,7 +126,21 @@ void free_subtree(Node* nd) {
 typedef std::tuple<u64, int64_t, int32_t> EvKey;
 EvKey ev_key(const Node* nd) { return EvKey(nd->last_use, -(int64_t)nd->depth, nd->block_id); }
 
+// One access to a node.  LRU (paper Section 1: least recently used blocks of finished requests go first): stamp
+// with the call's epoch.  GDSF (Section 4.1 "Access pattern-aware eviction policy": frequency beats recency for
+// prefixes; Greedy-Dual-Size-Frequency gives priority H = L + F * cost / size, L = priority of the last victim):
+// all blocks have one size and one cost here, so H = L + F.
+void touch(Oracle* o, Node* nd) {
+  if (o->policy == 0) { nd->last_use = o->epoch; return; }
+  nd->freq += 1;
+  nd->last_use = std::max(nd->last_use, o->inflation + nd->freq);
+}
+void note_victim(Oracle* o, const Node* nd) {
+  if (o->policy == 1) o->inflation = std::max(o->inflation, nd->last_use);
+}
+
 void remove_node(Oracle* o, Node* nd) {           // delete a leaf, give its id back (back of the ring)
+  note_victim(o, nd);
   o->by_id[nd->block_id] = nullptr;
   o->by_key.erase(nd->key);
   o->free_list[nd->tier].push_back(nd->block_id);
@@ -178,6 +195,7 @@ int drop_sorted(Oracle* o, int tier, int n, int32_t* victims) {
 }
 
 void demote_node(Oracle* o, Node* nd) {           // HBM -> host, node stays in the trie
+  note_victim(o, nd);
   int32_t old_id = nd->block_id;
   int32_t new_id = o->free_list[TIER_HOST].front();
   o->free_list[TIER_HOST].pop_front();
@@ -243,11 +261,14 @@ void* oracle_create(int32_t layers, int32_t heads, int32_t dim, int32_t elem_byt
   for (int32_t i = 0; i < hbm_blocks; ++i) o->free_list[0].push_back(i);                 // ascending ids
   for (int32_t i = 0; i < host_blocks; ++i) o->free_list[1].push_back(hbm_blocks + i);
   o->by_id.assign((size_t)hbm_blocks + host_blocks, nullptr);
-  o->collisions = 0; o->epoch = 0; o->status = 0;
+  o->collisions = 0; o->epoch = 0; o->status = 0; o->policy = 0; o->inflation = 0;
   o->root.parent = nullptr; o->root.depth = -1; o->root.block_id = -1; o->root.tier = -1;
-  o->root.refcount = 0; o->root.last_use = 0; o->root.key = root_key(salt); o->root.tag = 0;
+  o->root.refcount = 0; o->root.last_use = 0; o->root.freq = 0; o->root.key = root_key(salt); o->root.tag = 0;
   return o;
 }
+
+void oracle_set_policy(void* h, int32_t policy) { ((Oracle*)h)->policy = policy; }
+uint64_t oracle_inflation(void* h) { return ((Oracle*)h)->inflation; }
 
 void oracle_destroy(void* h) {
   Oracle* o = (Oracle*)h;
@@ -282,7 +303,7 @@ void oracle_lookup(void* h, const int32_t* tokens, const int64_t* off, int32_t R
       if (it == cur->children.end()) break;
       cur = it->second;
       ids[(int64_t)r * maxB + m] = cur->block_id;
-      if (!(flags & F_NO_TOUCH)) cur->last_use = o->epoch;
+      if (!(flags & F_NO_TOUCH)) touch(o, cur);
       if (flags & F_PIN) cur->refcount += 1;
     }
     for (int j = m; j < maxB; ++j) ids[(int64_t)r * maxB + j] = -1;
@@ -325,7 +346,7 @@ void oracle_insert(void* h, const int32_t* tokens, const int64_t* off, int32_t R
       auto it = cur->children.find(blk);
       if (it != cur->children.end()) {
         cur = it->second;
-        cur->last_use = o->epoch;
+        touch(o, cur);
         ids[(int64_t)r * maxB + j] = cur->block_id;
         continue;
       }
@@ -337,7 +358,7 @@ void oracle_insert(void* h, const int32_t* tokens, const int64_t* off, int32_t R
       o->free_list[TIER_HBM].pop_front();
       Node* nd = new Node();
       nd->parent = cur; nd->depth = j; nd->block_id = id; nd->tier = TIER_HBM; nd->refcount = 0;
-      nd->last_use = o->epoch; nd->key = chain_key(cur->key, content_hash(t, o->B));
+      nd->last_use = 0; nd->freq = 0; touch(o, nd); nd->key = chain_key(cur->key, content_hash(t, o->B));
       nd->tag = tags ? tags[(int64_t)r * maxB + j] : 0;
       nd->tokens = blk;
       if (o->by_key.count(nd->key)) o->collisions += 1; else o->by_key[nd->key] = nd;
@@ -446,14 +467,14 @@ int32_t oracle_live_count(void* h, int32_t tier) {
   for (Node* nd : o->by_id) if (nd && nd->tier == tier) ++c;
   return c;
 }
-// info[0..7] = live, refcount, last_use, depth, parent block id (-1 = root), key, tag, number of children
+// info[0..8] = live, refcount, last_use (stamp or priority), depth, parent block id (-1 = root), key, tag, number of children, freq
 void oracle_block_info(void* h, int32_t id, uint64_t* info) {
   Oracle* o = (Oracle*)h;
   Node* nd = (id >= 0 && id < (int32_t)o->by_id.size()) ? o->by_id[id] : nullptr;
-  if (!nd) { for (int i = 0; i < 8; ++i) info[i] = 0; return; }
+  if (!nd) { for (int i = 0; i < 9; ++i) info[i] = 0; return; }
   info[0] = 1; info[1] = (u64)nd->refcount; info[2] = nd->last_use; info[3] = (u64)nd->depth;
   info[4] = (u64)(int64_t)(nd->parent == &o->root ? -1 : nd->parent->block_id);
-  info[5] = nd->key; info[6] = nd->tag; info[7] = nd->children.size();
+  info[5] = nd->key; info[6] = nd->tag; info[7] = nd->children.size(); info[8] = nd->freq;
 }
 void oracle_block_tags(void* h, const int32_t* ids, int64_t n, uint64_t* out) {
   Oracle* o = (Oracle*)h;

@@ -44,6 +44,8 @@ def _load():
         lib.oracle_create.restype = vp
         lib.oracle_create.argtypes = [i32, i32, i32, i32, i32, u64, i32, i32, i32]
         lib.oracle_destroy.argtypes = [vp]
+        lib.oracle_set_policy.argtypes = [vp, i32]
+        lib.oracle_inflation.restype = u64; lib.oracle_inflation.argtypes = [vp]
         lib.oracle_hash.argtypes = [vp, vp, vp, i32, i32, vp]
         lib.oracle_lookup.argtypes = [vp, vp, vp, i32, i32, C.c_uint32, vp, vp]
         lib.oracle_fetch.argtypes = [vp, vp, vp, i32, i32, vp, u64, u64, C.c_uint32, vp]
@@ -88,7 +90,7 @@ def hash_parts():
 
 class Oracle:
     def __init__(self, layers, heads, dim, elem_bytes, block_tokens, salt, hbm_blocks, host_blocks=0,
-                 byte_mode=True):
+                 byte_mode=True, policy="lru"):
         self.lib = _load()
         self.layers, self.B = layers, block_tokens
         self.chunk_bytes = block_tokens * heads * dim * elem_bytes
@@ -97,6 +99,7 @@ class Oracle:
         self.byte_mode = byte_mode
         self.h = self.lib.oracle_create(layers, heads, dim, elem_bytes, block_tokens, salt, hbm_blocks,
                                         host_blocks, 1 if byte_mode else 0)
+        self.lib.oracle_set_policy(self.h, 1 if policy == "gdsf" else 0)
 
     def close(self):
         if self.h:
@@ -182,6 +185,9 @@ class Oracle:
     def epoch(self):
         return int(self.lib.oracle_epoch(self.h))
 
+    def inflation(self):
+        return int(self.lib.oracle_inflation(self.h))
+
     def collisions(self):
         return int(self.lib.oracle_collisions(self.h))
 
@@ -197,10 +203,10 @@ class Oracle:
         return int(self.lib.oracle_live_count(self.h, tier))
 
     def block_info(self, block_id):
-        info = np.zeros(8, dtype=np.uint64)
+        info = np.zeros(9, dtype=np.uint64)
         self.lib.oracle_block_info(self.h, int(block_id), _p(info))
         return dict(live=bool(info[0]), refcount=int(info[1]), last_use=int(info[2]), depth=int(info[3]),
-                    parent=int(np.int64(info[4])), key=int(info[5]), tag=int(info[6]), children=int(info[7]))
+                    parent=int(np.int64(info[4])), key=int(info[5]), tag=int(info[6]), children=int(info[7]), freq=int(info[8]))
 
     def block_tags(self, ids):
         ids = _i32(ids).ravel()

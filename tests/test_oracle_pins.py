@@ -555,3 +555,64 @@ def test_promotion_random_histories_keep_invariants_and_lookup_results():
             o.release(new_ids, m)
             check_invariants(o)
             o.evict(0, int(rng.integers(0, 6)), literal=bool(step % 2))
+
+
+# ---- frequency-aware eviction (GDSF with equal block size and cost) ---------------------------------------------
+def test_gdsf_keeps_frequent_blocks_that_lru_would_evict():
+    hot = np.array([1, 1, 2, 2], dtype=np.int32)           # two blocks, asked for five times early on
+    cold = np.array([7, 7, 8, 8], dtype=np.int32)          # two blocks, stored last, never asked for again
+    out = {}
+    for policy in ("lru", "gdsf"):
+        o = Oracle(1, 1, 8, 2, 2, 0, 8, policy=policy)
+        o.insert(*W.ragged([hot]), 2)                       # ids 0 1
+        for _ in range(5):
+            o.lookup(*W.ragged([hot]), 2)
+        o.insert(*W.ragged([cold]), 2)                      # ids 2 3, most recent
+        ne, v = o.evict(0, 2)
+        out[policy] = v.tolist()
+        if policy == "gdsf":
+            assert o.block_info(0)["freq"] == 6 and o.block_info(0)["last_use"] == 6     # H = L + F with L = 0
+            assert o.inflation() == 1                       # the victims had H = 0 + 1
+            o.insert(*W.ragged([cold]), 2)                  # re-stored after the eviction: H = L + 1 = 2; ids 4 5 (ring front)
+            assert o.block_info(4)["last_use"] == 2 and o.block_info(4)["freq"] == 1
+    assert out["lru"] == [1, 0]                             # least recently used: the hot pair goes
+    assert out["gdsf"] == [3, 2]                            # least frequently used: the cold pair goes, deeper first
+
+
+@pytest.mark.parametrize("host", [0, 40])
+def test_gdsf_literal_loop_equals_sorted_form_and_priorities_are_monotone(host):
+    for seed in range(40):
+        rng = np.random.default_rng(seed)
+        # a random script of serving steps, generated once and then run on two oracles
+        seqs, script = [], []
+        for step in range(30):
+            base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.7 else np.zeros(0, dtype=np.int32)
+            cut = int(rng.integers(0, len(base) + 1))
+            seqs.append(np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(2, 9)), dtype=np.int32)])[:20])
+            batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(int(rng.integers(1, 4)))] + [seqs[-1]]
+            script.append((batch, bool(rng.random() < 0.5), int(rng.integers(0, 2)) if host else 0, int(rng.integers(0, 12)),
+                           bool(rng.random() < 0.7)))
+        logs = []
+        for literal in (True, False):
+            o = Oracle(1, 1, 8, 2, 2, seed, 96, host, policy="gdsf")
+            log, held = [], []
+            for batch, pin, tier, n, release_now in script:
+                m, ids = o.lookup(*W.ragged(batch), 10, PIN if pin else 0)
+                l0 = o.inflation()
+                ne, v = o.evict(tier, n, literal=literal)
+                assert o.inflation() >= l0
+                ins, newb = o.insert(*W.ragged(batch), 10)
+                if pin:
+                    if release_now:
+                        o.release(ids, m)
+                    else:
+                        held.append((ids, m))
+                log.append((m.tolist(), ids.tolist(), ne.tolist(), v.tolist(), ins.tolist(), newb.tolist(), o.inflation(), o.status()))
+            nodes = all_nodes(o)
+            for i, nd in nodes.items():
+                if nd["parent"] >= 0:
+                    assert nodes[nd["parent"]]["last_use"] >= nd["last_use"]       # priority never rises towards the leaves
+                    assert nodes[nd["parent"]]["freq"] >= nd["freq"]
+                    assert nodes[nd["parent"]]["refcount"] >= nd["refcount"]
+            logs.append(log)
+        assert logs[0] == logs[1], seed
