@@ -142,7 +142,7 @@ class Serving:
         self.promote = args.promote if host_blocks else 0
         self.mb = self.stream.max_blocks
         flags = (G.COPY_BULK if args.engine == "bulk" else G.COPY_VECTOR) | G.copy_variant(args.variant) | \
-            G.copy_ctas_per_sm(args.ctas_per_sm)
+            G.copy_ctas_per_sm(args.ctas_per_sm) | (G.EVICT_GDSF if args.policy == "gdsf" else 0)
         self.store = G.PTStore(self.sh.layers, self.sh.heads, self.sh.dim, self.sh.block_tokens, self.pool_blocks,
                                max_requests=self.batch, max_batch_blocks=self.batch * self.mb, flags=flags, host_blocks=host_blocks)
         self.rng = np.random.default_rng(W.BASE_SEED + 77 + rank)
@@ -345,7 +345,7 @@ def run_gpu(args):
         "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8", "data": "synthetic",
         "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(wl.stream.docs),
-                   "batch": wl.batch, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
+                   "batch": wl.batch, "eviction": args.policy, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
                    "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
         "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_inserted": main["inserted"] / K, "blocks_dropped": main["dropped"] / K,
@@ -575,6 +575,7 @@ def main():
     ap.add_argument("--docs", type=int, default=0)
     ap.add_argument("--pool-blocks", type=int, default=0)
     ap.add_argument("--host-gb", type=float, default=0.0)
+    ap.add_argument("--policy", default="lru", choices=["lru", "gdsf"], help="eviction order")
     ap.add_argument("--promote", type=int, default=0, help="churn workload: host-tier blocks promoted into HBM per step (budget)")
     ap.add_argument("--lanes", type=int, default=0, help="lookup workload: lanes per request (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")

@@ -68,6 +68,11 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 /* flags of ptstore_config_t */
 #define PTSTORE_COPY_VECTOR  0x0u  /* copy engine: 16-byte vector loads/stores (always used for the host tier) */
 #define PTSTORE_COPY_BULK    0x1u  /* copy engine: bulk-async copies through a shared-memory ring (HBM<->HBM) */
+/* eviction order (Section 4.1 "Access pattern-aware eviction policy"): default is least recently used; with this
+ * flag it is Greedy-Dual-Size-Frequency with one size and one cost per block: priority H = L + F, F = accesses of
+ * the block (one per request that matched or stored it), L = the largest priority evicted so far.  Ties and the
+ * leaves-first rule are as for LRU. */
+#define PTSTORE_EVICT_GDSF   0x2u
 /* tuning fields of flags (0 = library default): lanes per request of the lookup (8, 16 or 32),
  * copy-kernel variant, copy CTAs per SM */
 #define PTSTORE_LOOKUP_LANES(n)   (((uint32_t)(n) & 0xFFu) << 8)
@@ -121,6 +126,7 @@ typedef struct {                 /* all counters are cumulative since create */
   uint64_t blocks_demoted;       /* HBM -> host */
   uint64_t rebuilds;
   uint64_t blocks_promoted;      /* host -> HBM */
+  uint64_t gdsf_clock;           /* GDSF policy: largest priority evicted so far */
 } ptstore_stats_t;
 
 /*

@@ -58,6 +58,7 @@ struct Ctrl {
   u64 blocks_demoted;
   u64 rebuilds;
   u64 blocks_promoted;
+  u64 inflation;        // GDSF clock L: largest priority evicted so far
   // lookup counters are striped so that thousands of warps do not queue on four addresses;
   // [stripe][0..3] = query blocks, probes issued, slots visited, blocks matched
   u64 lookup_stripes[LOOKUP_STRIPES][4];
@@ -70,7 +71,8 @@ struct Store {
   // per-block metadata, indexed by block id (both tiers)
   u64* m_key;           // 0 = block not live
   u64* m_parent;        // key of the parent node (root key for depth 0)
-  u64* m_last;          // LRU stamp
+  u64* m_last;          // LRU policy: stamp of the last touch; GDSF policy: priority H = L + F at the last touch
+  u32* m_freq;          // GDSF policy: access count F
   u32* m_ref;
   u32* m_depth;
   int* ring_ids[2];
@@ -81,6 +83,7 @@ struct Store {
   u32 layers;
   u32 block_tokens;
   u64 root_key;
+  u32 policy;           // 0 = LRU, 1 = GDSF (equal size and cost per block)
 };
 
 // ---- chained block hash -----------------------------------------------------------------------------
@@ -170,6 +173,15 @@ __device__ __forceinline__ unsigned char* block_ptr(const Store& st, u32 id) {
 }
 
 __device__ __forceinline__ void raise(const Store& st, u32 bit) { atomicOr(&st.ctrl->status, bit); }
+
+// `count` accesses to block `id` in the call with stamp `epoch` (paper Section 1: LRU; Section 4.1 "Access
+// pattern-aware eviction policy": frequency-aware Greedy-Dual-Size-Frequency, H = L + F * cost / size with
+// one size and one cost per block, so H = L + F; L = priority of the last victim, read once per kernel).
+__device__ __forceinline__ void touch_block(const Store& st, u32 id, u64 epoch, u64 inflation, u32 count) {
+  if (st.policy == 0) { st.m_last[id] = epoch; return; }
+  const u32 f = atomicAdd(&st.m_freq[id], count) + count;
+  atomicMax(&st.m_last[id], inflation + (u64)f);
+}
 
 // full blocks of request r, capped
 __device__ __forceinline__ int full_blocks(const long long* __restrict__ offsets, int r, u32 B, int max_blocks) {

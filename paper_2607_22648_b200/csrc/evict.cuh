@@ -195,9 +195,10 @@ __global__ void __launch_bounds__(256) apply_drop_kernel(Store st, int tier, con
   }
 }
 
-__global__ void drop_finish_kernel(Store st, int tier, int mode, int* __restrict__ n_evicted) {
+__global__ void drop_finish_kernel(Store st, int tier, int mode, const Key2* __restrict__ sorted, int* __restrict__ n_evicted) {
   Ctrl* c = st.ctrl;
   const u32 take = ev_take(c);
+  if (st.policy && take && sorted[take - 1].hi > c->inflation) c->inflation = sorted[take - 1].hi;   // GDSF clock
   c->ring[tier].count += take;
   c->live[tier] -= take;
   c->tombstones += take;
@@ -221,6 +222,7 @@ __global__ void __launch_bounds__(256) apply_demote_kernel(Store st, const Key2*
     st.m_key[new_id] = st.m_key[old_id];
     st.m_parent[new_id] = st.m_parent[old_id];
     st.m_last[new_id] = st.m_last[old_id];
+    st.m_freq[new_id] = st.m_freq[old_id];
     st.m_ref[new_id] = 0;
     st.m_depth[new_id] = st.m_depth[old_id];
     st.m_key[old_id] = 0;
@@ -230,8 +232,8 @@ __global__ void __launch_bounds__(256) apply_demote_kernel(Store st, const Key2*
   }
 }
 
-__global__ void __launch_bounds__(256) demote_finish_kernel(Store st, int* __restrict__ n_evicted, int* __restrict__ victims,
-                                                            const int* __restrict__ room_victims) {
+__global__ void __launch_bounds__(256) demote_finish_kernel(Store st, const Key2* __restrict__ sorted, int* __restrict__ n_evicted,
+                                                            int* __restrict__ victims, const int* __restrict__ room_victims) {
   Ctrl* c = st.ctrl;
   const u32 take = ev_take(c);
   const u32 dropped = c->ev_host_dropped;
@@ -246,6 +248,7 @@ __global__ void __launch_bounds__(256) demote_finish_kernel(Store st, int* __res
     c->live[1] += take;
     c->n_pairs = take;
     c->blocks_demoted += take;
+    if (st.policy && take && sorted[take - 1].hi > c->inflation) c->inflation = sorted[take - 1].hi;
     if (n_evicted) { n_evicted[0] = (int)take; n_evicted[1] = (int)dropped; }
   }
 }
@@ -287,7 +290,7 @@ __global__ void __launch_bounds__(256) table_rebuild_kernel(Store st, const Slot
 __global__ void __launch_bounds__(256) store_init_kernel(Store st) {
   const u32 total = st.n[0] + st.n[1];
   for (u32 i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-    st.m_key[i] = 0; st.m_parent[i] = 0; st.m_last[i] = 0; st.m_ref[i] = 0; st.m_depth[i] = 0;
+    st.m_key[i] = 0; st.m_parent[i] = 0; st.m_last[i] = 0; st.m_freq[i] = 0; st.m_ref[i] = 0; st.m_depth[i] = 0;
     if (i < st.n[0]) st.ring_ids[0][i] = (int)i;
     else st.ring_ids[1][i - st.n[0]] = (int)i;
   }

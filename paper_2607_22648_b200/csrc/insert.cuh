@@ -137,7 +137,8 @@ __global__ void __launch_bounds__(INS_THREADS) insert_assign_kernel(Store st, co
   const int j = (int)(e % max_blocks);
   st.m_key[id] = keys[e];
   st.m_parent[id] = j ? keys[e - 1] : st.root_key;
-  st.m_last[id] = epoch;
+  st.m_last[id] = st.policy ? 0 : epoch;      // GDSF: the finish kernel counts this call's accesses
+  st.m_freq[id] = 0;
   st.m_ref[id] = 0;
   st.m_depth[id] = (u32)j;
   slot->aux = NO_ID;
@@ -156,12 +157,13 @@ __global__ void __launch_bounds__(INS_THREADS) insert_assign_kernel(Store st, co
 
 __global__ void __launch_bounds__(256) insert_finish_kernel(Store st, const u32* __restrict__ eslot, long long total, u64 epoch,
                                                             int* __restrict__ ids_out) {
+  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
   for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
     const u32 s = eslot[e];
     int out = -1;
     if (s != NO_SLOT) {
       const u32 id = st.table[s].id;
-      if (id != NO_ID) { out = (int)id; st.m_last[id] = epoch; }
+      if (id != NO_ID) { out = (int)id; touch_block(st, id, epoch, inflation, 1); }
     }
     ids_out[e] = out;
   }

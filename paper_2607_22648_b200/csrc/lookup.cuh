@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
   const int nblk = valid ? full_blocks(offsets, (int)r, st.block_tokens, max_blocks) : 0;
   const long long tok0 = valid ? offsets[r] : 0;
   u64 parent = st.root_key;
+  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
   int m = 0;
   bool done = nblk == 0;
   u32 my_probes = 0, my_visited = 0;
@@ -103,10 +104,15 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
     const unsigned hm = __ballot_sync(FULL, hit);
     if (hit) {
       ids_out[r * max_blocks + j] = (int)id;
-      if (!(flags & F_NO_TOUCH)) st.m_last[id] = epoch;
-      if (flags & F_PIN) {
+      const bool touch = !(flags & F_NO_TOUCH);
+      if (touch && st.policy == 0) st.m_last[id] = epoch;
+      if ((flags & F_PIN) || (touch && st.policy)) {           // one atomic per distinct block in the warp
         const unsigned same = __match_any_sync(hm, id);
-        if (lane == __ffs(same) - 1) atomicAdd(&st.m_ref[id], (u32)__popc(same));
+        if (lane == __ffs(same) - 1) {
+          const u32 cnt = (u32)__popc(same);
+          if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
+          if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
+        }
       }
     }
     if (!done) {

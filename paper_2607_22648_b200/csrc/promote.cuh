@@ -118,6 +118,7 @@ __global__ void __launch_bounds__(INS_THREADS) promote_assign_kernel(Store st, c
   st.m_key[new_id] = st.m_key[old_id];
   st.m_parent[new_id] = st.m_parent[old_id];
   st.m_last[new_id] = st.m_last[old_id];
+  st.m_freq[new_id] = st.m_freq[old_id];
   st.m_ref[new_id] = st.m_ref[old_id];
   st.m_depth[new_id] = st.m_depth[old_id];
   st.m_key[old_id] = 0;

@@ -22,7 +22,7 @@ constexpr u64 ALIGN = 256;
 inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
-  u64 table[2], m_key, m_parent, m_last, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
+  u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
       cta_sums, prefix, promo_first, promo_cnt, total;
   u32 n_tiles;
 };
@@ -47,7 +47,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.table[0] = take(c->table_slots * sizeof(Slot));
   L.table[1] = take(c->table_slots * sizeof(Slot));
   L.m_key = take(N * 8); L.m_parent = take(N * 8); L.m_last = take(N * 8);
-  L.m_ref = take(N * 4); L.m_depth = take(N * 4);
+  L.m_freq = take(N * 4); L.m_ref = take(N * 4); L.m_depth = take(N * 4);
   L.ring[0] = take((u64)c->hbm_blocks * 4); L.ring[1] = take((u64)c->host_blocks * 4);
   L.ctrl = take(sizeof(Ctrl));
   L.blocked = take(N);
@@ -267,7 +267,8 @@ int launch_sort(ptstore* h, cudaStream_t s, int* result) {
   for (int b = 0; b < id_bytes; ++b) passes[np++] = {0, 8 * b};
   passes[np++] = {0, 32};
   passes[np++] = {0, 40};
-  const int st_bytes = bytes_needed(h->epoch);
+  // LRU: stamps are at most the epoch.  GDSF: a priority is at most the number of accesses ever counted
+  const int st_bytes = bytes_needed(h->st.policy ? h->epoch * (u64)h->cfg.max_requests : h->epoch);
   for (int b = 0; b < st_bytes; ++b) passes[np++] = {1, 8 * b};
   for (int p = 0; p < np; ++p) {
     sort_hist_kernel<<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
@@ -319,7 +320,7 @@ int run_drop(ptstore* h, int tier, int mode, u32 n, int* n_evicted, int* victims
   if (rc) return rc;
   apply_drop_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, tier, h->sort_buf[res], mode == EV_DROP ? victims : h->room);
   PTS_CHECK_LAUNCH(h);
-  drop_finish_kernel<<<1, 1, 0, s>>>(h->st, tier, mode, n_evicted);
+  drop_finish_kernel<<<1, 1, 0, s>>>(h->st, tier, mode, h->sort_buf[res], n_evicted);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
@@ -361,6 +362,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   st.m_key = reinterpret_cast<u64*>(w + lay.m_key);
   st.m_parent = reinterpret_cast<u64*>(w + lay.m_parent);
   st.m_last = reinterpret_cast<u64*>(w + lay.m_last);
+  st.m_freq = reinterpret_cast<u32*>(w + lay.m_freq);
   st.m_ref = reinterpret_cast<u32*>(w + lay.m_ref);
   st.m_depth = reinterpret_cast<u32*>(w + lay.m_depth);
   st.ring_ids[0] = reinterpret_cast<int*>(w + lay.ring[0]);
@@ -374,6 +376,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   st.layers = cfg->num_layers;
   st.block_tokens = cfg->block_tokens;
   st.root_key = hroot(cfg->salt);
+  st.policy = (cfg->flags & PTSTORE_EVICT_GDSF) ? 1u : 0u;
   h->blocked = w + lay.blocked;
   h->sort_buf[0] = reinterpret_cast<Key2*>(w + lay.sort[0]);
   h->sort_buf[1] = reinterpret_cast<Key2*>(w + lay.sort[1]);
@@ -530,7 +533,7 @@ int ptstore_evict(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evict
   if (rc) return rc;
   apply_demote_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, h->sort_buf[res], h->desc, victim_ids);
   PTS_CHECK_LAUNCH(h);
-  demote_finish_kernel<<<1, 256, 0, s>>>(h->st, n_evicted, victim_ids, h->room);
+  demote_finish_kernel<<<1, 256, 0, s>>>(h->st, h->sort_buf[res], n_evicted, victim_ids, h->room);
   PTS_CHECK_LAUNCH(h);
   Paged none = {};
   return launch_copy<COPY_POOL>(h, none, true, s);
@@ -614,6 +617,7 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
   out->blocks_demoted = c.blocks_demoted;
   out->rebuilds = c.rebuilds;
   out->blocks_promoted = c.blocks_promoted;
+  out->gdsf_clock = c.inflation;
   return PTSTORE_OK;
 }
 

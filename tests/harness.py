@@ -18,10 +18,12 @@ def dev(a, dtype=None):
 
 class Pair:
     def __init__(self, shape, hbm_blocks, host_blocks=0, salt=0, flags=0, max_requests=64, max_batch_blocks=4096,
-                 table_slots=None, byte_mode=True):
+                 table_slots=None, byte_mode=True, policy="lru"):
         self.shape = shape
+        if policy == "gdsf":
+            flags |= G.EVICT_GDSF
         self.o = Oracle(shape.layers, shape.heads, shape.dim, shape.elem_bytes, shape.block_tokens, salt, hbm_blocks,
-                        host_blocks, byte_mode=byte_mode)
+                        host_blocks, byte_mode=byte_mode, policy=policy)
         self.g = G.PTStore(shape.layers, shape.heads, shape.dim, shape.block_tokens, hbm_blocks, max_requests,
                            max_batch_blocks, elem_bytes=shape.elem_bytes, host_blocks=host_blocks, salt=salt, flags=flags,
                            table_slots=table_slots)
@@ -120,4 +122,5 @@ class Pair:
             assert s.live_nodes[t] == self.o.live_count(t), ("live", t, s.live_nodes[t], self.o.live_count(t))
             assert s.free_blocks[t] == self.o.free_count(t), ("free", t)
         assert s.epoch == self.o.epoch()
+        assert s.gdsf_clock == self.o.inflation()
         return s

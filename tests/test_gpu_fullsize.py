@@ -23,7 +23,8 @@ def _free_gb():
     return free / 1e9
 
 
-def test_llama8b_pool20k_batch64_serving_steps():
+@pytest.mark.parametrize("policy", ["lru", "gdsf"])
+def test_llama8b_pool20k_batch64_serving_steps(policy):
     """config 2 at full size: 20,000-block pool (39 GiB), 500 documents, 64 prompts per step."""
     from tests.serving import LockstepServing
     sh = W.LLAMA3_8B
@@ -32,7 +33,7 @@ def test_llama8b_pool20k_batch64_serving_steps():
     mb = st.max_blocks
     batches = [st.batch(64) for _ in range(5)]
     cache_blocks = max(sum(len(s) // sh.block_tokens for s in b[0]) for b in batches) + 8
-    srv = LockstepServing(sh, pool, 0, 64, mb, cache_blocks, seed=2)
+    srv = LockstepServing(sh, pool, 0, 64, mb, cache_blocks, seed=2, policy=policy)
     seen_evict = False
     for k, (seqs, tags) in enumerate(batches):
         r = srv.step(seqs, tags, sample=80, check_all=True, poison=(k == 3))

@@ -124,15 +124,16 @@ def test_insert_dedupe_denial_and_alloc_order():
     p.close()
 
 
-@pytest.mark.parametrize("host", [0, 24])
-def test_random_churn_lockstep(host):
+@pytest.mark.parametrize("host,policy", [(0, "lru"), (24, "lru"), (0, "gdsf"), (24, "gdsf")])
+def test_random_churn_lockstep(host, policy):
     """Random interleaving of lookup(PIN) / fetch / evict / insert / release, compared call by call."""
     Pair, dev, G = _imports()
     sh = W.KVShape(2, 1, 8, 2)
     B = 2
     for seed in range(6):
         rng = np.random.default_rng(100 + seed)
-        p = Pair(sh, 40, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * 12, table_slots=211 if seed % 2 else 401)
+        p = Pair(sh, 40, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * 12, table_slots=211 if seed % 2 else 401,
+                 policy=policy)
         seqs, pinned = [], []
         for step in range(60):
             base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.75 else np.zeros(0, dtype=np.int32)
@@ -212,6 +213,27 @@ def test_promotion_worked_example_and_unpinned_lists():
     with pytest.raises(G.PTStoreError):
         Pair(sh, 8).g.promote(dev(io3), dev(mo3), 0, 1)          # no host tier
     p.close()
+
+
+def test_gdsf_keeps_frequent_blocks_that_lru_would_evict():
+    Pair, dev, G = _imports()
+    hot = np.array([1, 1, 2, 2], dtype=np.int32)
+    cold = np.array([7, 7, 8, 8], dtype=np.int32)
+    out = {}
+    for policy in ("lru", "gdsf"):
+        p = Pair(W.KVShape(1, 1, 8, 2), 8, max_requests=4, max_batch_blocks=16, policy=policy)
+        p.insert([hot], 2)
+        for _ in range(5):
+            p.lookup([hot, hot[:2]], 2)                      # two requests per call touch the first block
+        p.insert([cold], 2)
+        ne, v = p.evict(0, 2)
+        out[policy] = v.tolist()
+        p.insert([cold, cold], 2)
+        p.lookup([hot, cold], 2, flags=1)
+        p.evict(0, 8)
+        p.check_counts()
+        p.close()
+    assert out["lru"] == [1, 0] and out["gdsf"] == [3, 2]
 
 
 def test_lookup_stress_small_matches_oracle():
