@@ -117,10 +117,18 @@ class Serving:
         free_gb = torch.cuda.mem_get_info()[0] / 1e9
         host_blocks = 0
         if kind == "llama8b":
+            bt = args.block_tokens or 16
+            self.sh = W.KVShape(32, 8, 128, bt)
+            self.batch, self.pool_blocks = args.batch or 64, args.pool_blocks or 20000 * 16 // bt
+            self.stream = W.llama8b_stream(seed=W.BASE_SEED + 1 + 1000 * rank, n_docs=args.docs or 500, shape=self.sh)
+            self.name = "llama3_8b_kv_pool%dk_zipf1.1_batch%d" % (self.pool_blocks // 1000, self.batch) if bt == 16 else \
+                "llama3_8b_kv_block%d_pool%d_zipf1.1_batch%d" % (bt, self.pool_blocks, self.batch)
+            self.kv = "32L x 8H x 128 bf16, block %d" % bt
+        elif kind == "multiturn":
             self.sh = W.LLAMA3_8B
             self.batch, self.pool_blocks = args.batch or 64, args.pool_blocks or 20000
-            self.stream = W.llama8b_stream(seed=W.BASE_SEED + 1 + 1000 * rank, n_docs=args.docs or 500)
-            self.name = "llama3_8b_kv_pool%dk_zipf1.1_batch%d" % (self.pool_blocks // 1000, self.batch)
+            self.stream = W.conversation_stream(seed=W.BASE_SEED + 5 + 1000 * rank, n_conversations=args.docs or 512)
+            self.name = "multiturn_llama3_8b_kv_pool%d_conv%d_batch%d" % (self.pool_blocks, self.stream.n_conversations, self.batch)
             self.kv = "32L x 8H x 128 bf16, block 16"
         elif kind == "llama70b":
             self.sh = W.LLAMA3_70B
@@ -344,7 +352,7 @@ def run_gpu(args):
         "metric": "prefix-hit KV fetch GB/s", "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W_,
         "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8", "data": "synthetic",
-        "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(wl.stream.docs),
+        "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(getattr(wl.stream, "docs", ())) or wl.stream.n_conversations,
                    "batch": wl.batch, "eviction": args.policy, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
                    "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
@@ -570,7 +578,8 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--fill", type=int, default=6, help="untimed steps that fill the pool before warm-up")
-    ap.add_argument("--workload", default="llama8b", choices=["llama8b", "llama70b", "churn", "lookup"])
+    ap.add_argument("--workload", default="llama8b", choices=["llama8b", "llama70b", "churn", "lookup", "multiturn"])
+    ap.add_argument("--block-tokens", type=int, default=0, help="llama8b workload: tokens per block (default 16)")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--docs", type=int, default=0)
     ap.add_argument("--pool-blocks", type=int, default=0)

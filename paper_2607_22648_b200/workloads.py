@@ -284,3 +284,55 @@ def lookup_stress(seed=BASE_SEED + 2, n_roots=50000, trunk=12, branch=4, n_queri
         depth[q] = d
     n_nodes = n_roots * (trunk + 2 * branch)
     return LookupStress(B, store, queries, depth, n_nodes, int(np.ceil(n_nodes / load)), vocab)
+
+
+# ---------------------------------------------------------------------------------------------------
+# multi-turn conversations: growing chains, deep tries, small increments
+# ---------------------------------------------------------------------------------------------------
+@dataclass
+class ConversationStream:
+    """Each conversation is an append-only token sequence; a request is the whole history plus a new turn, so
+    all earlier full blocks are a stored prefix and every step adds only a few blocks per conversation."""
+    shape: KVShape
+    n_conversations: int
+    turn_range: tuple
+    max_tokens: int
+    vocab: int
+    seed: int
+    rng: np.random.Generator = field(repr=False, default=None)
+    history: list = field(repr=False, default_factory=list)
+
+    @property
+    def max_blocks(self):
+        return -(-self.max_tokens // self.shape.block_tokens)
+
+    def batch(self, n_requests):
+        """-> (seqs, tags) for n_requests distinct conversations, each extended by one turn (a conversation that
+        would outgrow max_tokens starts over with a fresh id)."""
+        B = self.shape.block_tokens
+        pick = self.rng.choice(self.n_conversations, size=min(n_requests, self.n_conversations), replace=False)
+        seqs, tags = [], []
+        for c in pick:
+            uid, toks = self.history[c]
+            turn = self.rng.integers(0, self.vocab, size=int(self.rng.integers(self.turn_range[0], self.turn_range[1] + 1)),
+                                     dtype=np.int32)
+            if len(toks) + len(turn) > self.max_tokens:
+                uid, toks = self._fresh_uid(), np.zeros(0, dtype=np.int32)
+            toks = np.concatenate([toks, turn])
+            self.history[c] = (uid, toks)
+            nb = len(toks) // B
+            seqs.append(toks)
+            tags.append((np.uint64(uid) << np.uint64(24)) | np.arange(nb, dtype=np.uint64))
+        return seqs, tags
+
+    def _fresh_uid(self):
+        self._next = getattr(self, "_next", 0) + 1
+        return (1 << 28) + self._next
+
+
+def conversation_stream(seed=BASE_SEED + 5, shape=LLAMA3_8B, n_conversations=256, turn_range=(50, 400), max_tokens=8192,
+                        vocab=128256):
+    st = ConversationStream(shape, n_conversations, turn_range, max_tokens, vocab, seed,
+                            np.random.Generator(np.random.PCG64(seed)))
+    st.history = [(st._fresh_uid(), np.zeros(0, dtype=np.int32)) for _ in range(n_conversations)]
+    return st

@@ -128,3 +128,44 @@ def test_churn_with_host_tier():
     print("churn: hbm %d blocks, host %d blocks (%.0f GB pinned), %d steps, demoted %d, host drops %d, promoted %d, fetched from hbm/host %s"
           % (hbm, host, host * sh.block_bytes / 1e9, n_steps, demoted, dropped, promoted, srv.fetched_by_tier))
     srv.close()
+
+
+def test_multi_turn_conversations_grow_chains_by_small_increments():
+    """A second workload shape: 256 append-only conversations, 32 of them extended per step; every step matches the
+    whole stored history and adds a few blocks per request; the pool turns over through LRU eviction."""
+    from tests.serving import LockstepServing
+    sh = W.LLAMA3_8B
+    st = W.conversation_stream(n_conversations=256, max_tokens=4096)
+    mb = st.max_blocks
+    srv = LockstepServing(sh, 5000, 0, 32, mb, 32 * mb, seed=6)
+    hits = evicts = 0
+    for k in range(40):
+        seqs, tags = st.batch(32)
+        r = srv.step(seqs, tags, sample=8, check_all=(k % 8 == 7))
+        hits += r["matched"]
+        evicts += r["evicted"] is not None
+        assert r["status"] == 0
+    s = srv.check_counts()
+    assert srv.check_pool(32) > 0
+    assert hits > 5000 and evicts > 0 and srv.sampled_chunks >= 256
+    print("multi-turn: matched %d blocks over 40 steps, %d steps evicted, live %d" % (hits, evicts, s.live_nodes[0]))
+    srv.close()
+
+
+def test_large_blocks_of_1024_tokens():
+    """The block size the paper quotes for its vLLM baseline (1024 tokens): 2 MiB chunks, 128 MiB blocks."""
+    from tests.serving import LockstepServing
+    sh = W.KVShape(32, 8, 128, 1024)
+    st = W.doc_stream(W.BASE_SEED + 6, sh, n_docs=40, len_range=(2000, 6000), zipf_s=1.1, vocab=128256, suffix_range=(64, 256))
+    mb = st.max_blocks
+    srv = LockstepServing(sh, 64, 0, 8, mb, 8 * mb, seed=7)
+    matched = 0
+    for k in range(8):
+        seqs, tags = st.batch(8)
+        r = srv.step(seqs, tags, sample=40, check_all=True)
+        matched += r["matched"]
+    srv.check_counts()
+    assert srv.check_pool(8) > 0
+    assert matched > 20 and srv.sampled_chunks >= 256
+    print("1024-token blocks: chunk %d KiB, block %d MiB, matched %d blocks" % (sh.chunk_bytes >> 10, sh.block_bytes >> 20, matched))
+    srv.close()
