@@ -127,6 +127,8 @@ typedef struct {                 /* all counters are cumulative since create */
   uint64_t rebuilds;
   uint64_t blocks_promoted;      /* host -> HBM */
   uint64_t gdsf_clock;           /* GDSF policy: largest priority evicted so far */
+  uint64_t blocks_fetched_distinct; /* distinct source blocks read by fetch calls: a block named by several requests
+                                       of one call is read once and written to each destination */
 } ptstore_stats_t;
 
 /*
@@ -178,6 +180,7 @@ int ptstore_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets,
  * the application supplies).  For every r, j < matched_blocks[r], layer l, s in {K,V}: copy one chunk
  * from pool block block_ids[r*max_blocks+j] to block block_tables[r*max_blocks+j] of the paged cache.
  * Host-tier blocks are read in place through the mapped pointer.  No metadata changes.
+ * A pool block named by several entries of the call is read once and written to every destination.
  * Entries with an id or table entry out of range are skipped and raise S_BOUNDS.
  */
 int ptstore_fetch(ptstore_t* st, const int32_t* block_ids, const int32_t* matched_blocks, int32_t R,

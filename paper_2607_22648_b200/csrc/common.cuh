@@ -49,7 +49,7 @@ struct Ctrl {
   u32 ev_host_dropped;  // evict: host-tier drops that made room for a demotion
   u32 live[2];
   u32 tombstones;
-  u32 pad1;
+  u32 work_counter;     // fetch: next work unit to hand out (dynamic dealing inside the copy kernel)
   // cumulative counters
   u64 query_blocks, probes_issued, slots_visited, blocks_matched;   // totals are these plus the stripes below
   u64 blocks_fetched[2];
@@ -59,6 +59,7 @@ struct Ctrl {
   u64 rebuilds;
   u64 blocks_promoted;
   u64 inflation;        // GDSF clock L: largest priority evicted so far
+  u64 blocks_fetched_distinct;   // distinct source blocks read by fetch calls (<= blocks fetched)
   // lookup counters are striped so that thousands of warps do not queue on four addresses;
   // [stripe][0..3] = query blocks, probes issued, slots visited, blocks matched
   u64 lookup_stripes[LOOKUP_STRIPES][4];

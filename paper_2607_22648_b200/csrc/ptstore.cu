@@ -23,7 +23,7 @@ inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
   u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
-      cta_sums, prefix, promo_first, promo_cnt, total;
+      cta_sums, prefix, promo_first, promo_cnt, links, total;
   u32 n_tiles;
 };
 
@@ -62,6 +62,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.prefix = take(((u64)c->max_requests + 1) * 4);
   L.promo_first = take(N * 4);
   L.promo_cnt = take(N * 4);
+  L.links = take(M * sizeof(int2));
   L.total = o;
   return L;
 }
@@ -86,11 +87,13 @@ struct ptstore {
   u32* prefix;
   u32* promo_first;
   u32* promo_cnt;
+  int2* links;           // fetch: destination list nodes, one per (request, block) entry
   u64 epoch;
   u64 launches;
   int last_cuda;
   int sms;
-  int bulk_smem_set[3];  // dynamic shared memory already granted to the bulk kernel of each mode
+  int bulk_smem_set[4];
+  int bulk_multi_smem_set;  // dynamic shared memory already granted to the bulk kernel of each mode
   bool has_env_tune;
   BulkVariant env_tune;
 };
@@ -225,6 +228,25 @@ int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, const BulkVariant& 
   return PTSTORE_OK;
 }
 
+// multi-destination fetch: dynamic dealing of `group`-piece units (default: a quarter of a source block)
+int launch_bulk_multi(ptstore* h, const Paged& pc, cudaStream_t s, BulkVariant v, int ctas_per_sm) {
+  const int smem = v.stages * v.stage_bytes;
+  if (smem > h->bulk_multi_smem_set) {
+    if (cudaFuncSetAttribute(copy_bulk_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      h->last_cuda = (int)cudaGetLastError();
+      return PTSTORE_E_CUDA;
+    }
+    h->bulk_multi_smem_set = smem;
+  }
+  const u32 ppc = (u32)((h->st.chunk_bytes + v.stage_bytes - 1) / v.stage_bytes);
+  const u32 per_pair = 2u * h->st.layers * ppc;
+  int group = v.group > 1 ? v.group : (int)(per_pair >= 4 ? per_pair / 4 : per_pair);
+  BulkTune t = {v.stages, v.stage_bytes, group, 0};
+  copy_bulk_multi_kernel<<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs, &h->st.ctrl->work_counter, t);
+  PTS_CHECK_LAUNCH(h);
+  return PTSTORE_OK;
+}
+
 template <int MODE>
 int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream_t s) {
   const u32 variant = (h->cfg.flags >> 16) & 0xFu;
@@ -233,6 +255,7 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
     BulkVariant v = kBulkVariants[variant < (u32)kNumBulkVariants ? variant : 0];
     if (v.stages == 0) v = auto_bulk(h->st.chunk_bytes);
     if (h->has_env_tune) v = h->env_tune;
+    if (MODE == COPY_FETCH_MULTI && !v.hint) return launch_bulk_multi(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm);
     return launch_bulk<MODE>(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm);
   }
   switch (variant) {
@@ -389,6 +412,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->prefix = reinterpret_cast<u32*>(w + lay.prefix);
   h->promo_first = reinterpret_cast<u32*>(w + lay.promo_first);
   h->promo_cnt = reinterpret_cast<u32*>(w + lay.promo_cnt);
+  h->links = reinterpret_cast<int2*>(w + lay.links);
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int cap = sms * 8;
@@ -451,12 +475,18 @@ int ptstore_fetch(ptstore_t* h, const int32_t* block_ids, const int32_t* matched
   rc = check_cache(h, dst);
   if (rc) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  scan_matched_kernel<<<1, 1024, 0, s>>>(h->st, matched_blocks, R, max_blocks, h->prefix);
+  // one descriptor per distinct source block, each with the list of its destinations (promo_first doubles as the list heads)
+  const u32 n_blocks = h->cfg.hbm_blocks + h->cfg.host_blocks;
+  const int cap = h->sms * 8;
+  fetch_begin_kernel<<<grid_for(n_blocks, 256, cap), 256, 0, s>>>(h->st, h->promo_first, n_blocks);
   PTS_CHECK_LAUNCH(h);
-  build_pairs_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, block_ids, matched_blocks, block_tables,
-                                                                                         R, max_blocks, dst->num_blocks, h->prefix, h->desc);
+  fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, block_tables, R, max_blocks,
+                                                                                 dst->num_blocks, h->promo_first, h->links, h->desc);
   PTS_CHECK_LAUNCH(h);
-  return launch_copy<COPY_FETCH>(h, to_paged(dst), h->cfg.host_blocks > 0, s);
+  Paged pc = to_paged(dst);
+  pc.head = h->promo_first;
+  pc.node = h->links;
+  return launch_copy<COPY_FETCH_MULTI>(h, pc, h->cfg.host_blocks > 0, s);
 }
 
 int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
@@ -618,6 +648,7 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
   out->rebuilds = c.rebuilds;
   out->blocks_promoted = c.blocks_promoted;
   out->gdsf_clock = c.inflation;
+  out->blocks_fetched_distinct = c.blocks_fetched_distinct;
   return PTSTORE_OK;
 }
 
