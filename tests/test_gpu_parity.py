@@ -378,3 +378,76 @@ def test_table_rebuild_under_delete_heavy_churn():
     s = p.check_counts()
     assert s.rebuilds > 0
     p.close()
+
+
+@pytest.mark.parametrize("name,mk", [ENGINES[0], ENGINES[3], ENGINES[4]], ids=["vector", "bulk", "bulk_8x8k_3cta"])
+def test_many_requests_share_one_prefix(name, mk):
+    """40 identical prompts: every pool block has 40 destinations (more than the per-unit destination cache holds),
+    plus a few prompts that share only the front of the prefix."""
+    Pair, dev, G = _imports()
+    sh = W.TINY
+    B = sh.block_tokens
+    rng = np.random.default_rng(9)
+    doc = rng.integers(0, 32000, size=20 * B + 5, dtype=np.int32)
+    other = np.concatenate([doc[:7 * B], rng.integers(0, 32000, size=6 * B, dtype=np.int32)])
+    p = Pair(sh, 64, flags=mk(G), max_requests=64, max_batch_blocks=64 * 24)
+    src = W.random_kv_cache(4, sh, 40)
+    p.insert([doc, other], 24, src, W.shuffled_block_tables(rng, [doc, other], B, 24, 40))
+    batch = [doc] * 40 + [other] * 3 + [doc[: 3 * B + 1]]
+    mo, io, _, _ = p.lookup(batch, 24, flags=1)
+    assert mo.tolist() == [20] * 40 + [13] * 3 + [3]
+    nd = int(mo.sum()) + 7
+    dst = [np.full((2, nd, sh.chunk_bytes), 0x11, dtype=np.uint8) for _ in range(sh.layers)]
+    bt = np.full((len(batch), 24), -1, dtype=np.int32)
+    perm, k = rng.permutation(nd), 0
+    for r in range(len(batch)):
+        for j in range(mo[r]):
+            bt[r, j] = perm[k]
+            k += 1
+    p.fetch(io, mo, dst, bt)
+    s = p.check_counts()
+    assert s.blocks_fetched[0] == int(mo.sum()) and s.blocks_fetched_distinct == 26      # 20 + 6 distinct source blocks
+    p.release(io, mo)
+    assert p.check_status() == 0
+    p.close()
+
+
+def test_degenerate_shapes():
+    Pair, dev, G = _imports()
+    rng = np.random.default_rng(3)
+    # a pool of one block, one block per request
+    p = Pair(W.KVShape(1, 1, 8, 1), 1, max_requests=4, max_batch_blocks=4, table_slots=3)
+    src = W.random_kv_cache(0, W.KVShape(1, 1, 8, 1), 4)
+    p.insert([np.array([5], dtype=np.int32), np.array([6], dtype=np.int32)], 1, src, np.array([[0], [1]], dtype=np.int32))
+    assert p.check_status() == G.S_NOSPACE
+    mo, io, _, _ = p.lookup([np.array([5, 6], dtype=np.int32), np.array([6], dtype=np.int32)], 1)
+    assert mo.tolist() == [1, 0]
+    p.evict(0, 1)
+    p.insert([np.array([6], dtype=np.int32)], 1, src, np.array([[2]], dtype=np.int32))
+    p.check_pools(); p.check_counts(); p.check_status()
+    p.close()
+    # one very long request: hundreds of chained chunks per warp, max_blocks in the thousands
+    sh = W.KVShape(1, 1, 8, 1)
+    p = Pair(sh, 6000, max_requests=4, max_batch_blocks=4 * 5000, byte_mode=False)
+    long_seq = rng.integers(0, 1000, size=5000, dtype=np.int32)
+    p.hash([long_seq, long_seq[:4321]], 5000)
+    p.insert([long_seq[:4000]], 5000)
+    mo, io, _, _ = p.lookup([long_seq, long_seq[:1234], np.concatenate([long_seq[:77], long_seq[:50]])], 5000, flags=1)
+    assert mo.tolist() == [4000, 1234, 77]
+    p.release(io, mo)
+    ne, v = p.evict(0, 1500)
+    assert ne[0] == 1500 and v[0] == 3999 and v[-1] == 2500
+    p.lookup([long_seq], 5000)
+    p.check_counts(); assert p.check_status() == 0
+    p.close()
+    # very many short requests
+    p = Pair(sh, 30000, max_requests=20000, max_batch_blocks=20000 * 2, byte_mode=False)
+    many = [rng.integers(0, 150, size=int(rng.integers(0, 3)), dtype=np.int32) for _ in range(20000)]
+    p.insert(many, 2)
+    mo, io, _, _ = p.lookup(many[::-1], 2, flags=1)
+    assert (mo == np.array([len(x) for x in many[::-1]])).all()
+    p.release(io, mo)
+    p.evict(0, 12345)
+    p.lookup(many, 2)
+    p.check_counts(); assert p.check_status() == 0
+    p.close()
