@@ -149,6 +149,7 @@ class Serving:
             self.kv = "32L x 8H x 128 bf16, block 16"
         self.host_blocks = host_blocks
         self.promote = args.promote if host_blocks else 0
+        self.async_demote = bool(args.async_demote and host_blocks)
         self.mb = self.stream.max_blocks
         flags = (G.COPY_BULK if args.engine == "bulk" else G.COPY_VECTOR) | G.copy_variant(args.variant) | \
             G.copy_ctas_per_sm(args.ctas_per_sm) | (G.EVICT_GDSF if args.policy == "gdsf" else 0)
@@ -208,22 +209,15 @@ class Serving:
             st.promote(self.ids, self.matched, G.PINNED_LIST, self.promote, self.nprom)
             if events is not None:
                 events["promote"][-1] = (events["promote"][-1][0], self._ev())
+        if self.async_demote:
+            self._evict_shortfall(s, events)          # its demotion copy (device -> host) overlaps the fetch (host -> device)
         if events is not None:
             events["fetch"].append((self._ev(), None))
         st.fetch(self.ids, self.matched, self.cache, d["bt"])
         if events is not None:
             events["fetch"][-1] = (events["fetch"][-1][0], self._ev())
-        # the serving engine needs the matched lengths on the host anyway; the same sync gives the free count
-        self.h_matched.copy_(self.matched, non_blocking=True)
-        stats = st.stats()
-        need = s["total_blocks"] - int(self.h_matched.sum()) + self.promote      # keep room for the next step's promotions
-        short = need - int(stats.free_blocks[0])
-        if short > 0:
-            if events is not None:
-                events["evict"].append((self._ev(), None))
-            st.evict(G.TIER_HBM, short, want_victims=False, n_evicted=self.nev)
-            if events is not None:
-                events["evict"][-1] = (events["evict"][-1][0], self._ev())
+        if not self.async_demote:
+            self._evict_shortfall(s, events)
         if events is not None:
             events["insert"].append((self._ev(), None))
         st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb)
@@ -233,6 +227,20 @@ class Serving:
         if e2e:
             self.h_ids.copy_(self.ids, non_blocking=True)
             self.h_newb.copy_(self.newb, non_blocking=True)
+
+    def _evict_shortfall(self, s, events):
+        # the serving engine needs the matched lengths on the host anyway; the same sync gives the free count
+        torch, G, st = self.torch, self.G, self.store
+        self.h_matched.copy_(self.matched, non_blocking=True)
+        stats = st.stats()
+        need = s["total_blocks"] - int(self.h_matched.sum()) + self.promote      # keep room for the next step's promotions
+        short = need - int(stats.free_blocks[0])
+        if short > 0:
+            if events is not None:
+                events["evict"].append((self._ev(), None))
+            st.evict(G.TIER_HBM, short, want_victims=False, n_evicted=self.nev, asynchronous=self.async_demote)
+            if events is not None:
+                events["evict"][-1] = (events["evict"][-1][0], self._ev())
 
     def _ev(self):
         e = self.torch.cuda.Event(enable_timing=True)
@@ -596,6 +604,7 @@ def main():
     ap.add_argument("--pool-blocks", type=int, default=0)
     ap.add_argument("--host-gb", type=float, default=0.0)
     ap.add_argument("--policy", default="lru", choices=["lru", "gdsf"], help="eviction order")
+    ap.add_argument("--async-demote", action="store_true", help="churn workload: evict before fetch with ptstore_evict_async")
     ap.add_argument("--promote", type=int, default=0, help="churn workload: host-tier blocks promoted into HBM per step (budget)")
     ap.add_argument("--lanes", type=int, default=0, help="lookup workload: lanes per request (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")

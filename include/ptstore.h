@@ -230,6 +230,23 @@ int ptstore_evict(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evic
                   ptstore_stream_t stream);
 
 /*
+ * ptstore_evict with the demotion copy (HBM -> host) on a stream of the library's own, so that it can share the
+ * host link, which is full duplex, with a fetch of host-tier blocks running the other way (the paper overlaps its
+ * transfers with computation, Section 4.1 "Fine-grain multi-level caching": data transfers happen asynchronously).
+ * Everything else is as for ptstore_evict: the metadata changes and both outputs are ordered on `stream`.
+ * The copy is ordered after them and before any later ptstore_insert, ptstore_promote, ptstore_evict[_async] and
+ * ptstore_join on this handle.  It is NOT ordered with later ptstore_fetch calls: until the next of the calls just
+ * named, fetch only block ids that were pinned (ptstore_lookup with PTSTORE_PIN) before this call — a pinned block
+ * is never a victim, so such a fetch cannot touch a block in flight.  Without a host tier, or for tier HOST, this
+ * is ptstore_evict.  The first call creates the stream and two events (no device memory).
+ */
+int ptstore_evict_async(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids,
+                        ptstore_stream_t stream);
+
+/* Make `stream` wait for a demotion copy left running by ptstore_evict_async (no-op if there is none). */
+int ptstore_join(ptstore_t* st, ptstore_stream_t stream);
+
+/*
  * Move host-tier blocks named by a batch into HBM (the paper keeps hot prefixes on the fastest tier, Section 4.1
  * "Replication of popular prefixes to improve access locality"; with one store the analogue is promoting a block
  * that was just hit).  Entries (r, j < matched_blocks[r]) are taken in (r, j) order, so the front of a prefix

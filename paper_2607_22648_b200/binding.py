@@ -57,7 +57,7 @@ class Stats(C.Structure):
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
-           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote"]
+           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join"]
 
 
 def _load():
@@ -76,6 +76,8 @@ def _load():
     lib.ptstore_insert.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
     lib.ptstore_release.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.ptstore_evict.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.ptstore_evict_async.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.ptstore_join.argtypes = [vp, vp]
     lib.ptstore_promote.argtypes = [vp, vp, vp, i32, i32, u32, i32, vp, vp]
     lib.ptstore_status.argtypes = [vp, vp, C.POINTER(u32)]
     lib.ptstore_stats.argtypes = [vp, vp, C.POINTER(Stats)]
@@ -138,7 +140,9 @@ class PTStore:
     """One store on one GPU.  Allocates pool and workspace with torch and hands them to the library."""
 
     def __init__(self, layers, heads, dim, block_tokens, hbm_blocks, max_requests, max_batch_blocks, elem_bytes=2,
-                 host_blocks=0, table_slots=None, salt=0, flags=0, device=0, hbm_pool=None, host_pool=None):
+                 host_blocks=0, table_slots=None, salt=0, flags=0, device=None, hbm_pool=None, host_pool=None):
+        if device is None:
+            device = torch.cuda.current_device()       # one process per GPU: the rank's own device
         self.device = torch.device("cuda", device)
         self.layers, self.block_tokens = layers, block_tokens
         self.chunk_bytes = block_tokens * heads * dim * elem_bytes
@@ -224,13 +228,17 @@ class PTStore:
         R, mb = ids.shape
         self._check(lib.ptstore_release(self.h, _ptr(ids), _ptr(matched), R, mb, _stream()), "ptstore_release")
 
-    def evict(self, tier, n, want_victims=True, n_evicted=None, victims=None):
+    def evict(self, tier, n, want_victims=True, n_evicted=None, victims=None, asynchronous=False):
         if n_evicted is None:
             n_evicted = torch.zeros(2, dtype=torch.int32, device=self.device)
         if victims is None and want_victims:
             victims = torch.full((max(2 * n, 1),), -1, dtype=torch.int32, device=self.device)
-        self._check(lib.ptstore_evict(self.h, tier, n, _ptr(n_evicted), _ptr(victims), _stream()), "ptstore_evict")
+        fn = lib.ptstore_evict_async if asynchronous else lib.ptstore_evict
+        self._check(fn(self.h, tier, n, _ptr(n_evicted), _ptr(victims), _stream()), "ptstore_evict")
         return n_evicted, victims
+
+    def join(self):
+        self._check(lib.ptstore_join(self.h, _stream()), "ptstore_join")
 
     def promote(self, ids, matched, flags, max_promote, n_promoted=None):
         """Rewrites `ids` in place; returns the device counter of blocks moved."""

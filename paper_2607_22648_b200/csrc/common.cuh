@@ -39,7 +39,9 @@ struct Ctrl {
   u32 status;
   u32 pad0;
   // per-call scalars produced by one kernel and consumed by the next
-  u32 n_pairs;          // fetch / release / insert / demote: entries in the copy descriptor list
+  u32 n_pairs;          // fetch / insert / promote: entries in the copy descriptor list
+  u32 n_pairs_host;     // fetch: distinct host-tier source blocks (their descriptors form a list of their own)
+  u32 n_pairs_tier;     // demotion: entries in its own descriptor list (its copy may run on the library's side stream)
   u32 ins_total_new;    // insert: new unique nodes presented
   u32 ins_granted;      // insert: of those, how many got a block
   u32 ins_base;         // insert: ring head before this call

@@ -491,14 +491,17 @@ __global__ void __launch_bounds__(256) build_pairs_kernel(Store st, const int* _
 // ---- destination lists for COPY_FETCH_MULTI ---------------------------------------------------------------------
 __global__ void __launch_bounds__(256) fetch_begin_kernel(Store st, u32* __restrict__ head, u32 n_blocks) {
   for (u32 i = blockIdx.x * blockDim.x + threadIdx.x; i < n_blocks; i += gridDim.x * blockDim.x) head[i] = LINK_NIL;
-  if (blockIdx.x == 0 && threadIdx.x == 0) { st.ctrl->n_pairs = 0; st.ctrl->work_counter = 0; }
+  if (blockIdx.x == 0 && threadIdx.x == 0) { st.ctrl->n_pairs = 0; st.ctrl->n_pairs_host = 0; st.ctrl->work_counter = 0; }
 }
 
 // every (r, j < matched[r]) entry pushes {cache block} on the list of its source block; the entry that finds the
-// list empty also appends the block to the descriptor list (one descriptor per distinct source block)
+// list empty also appends the block to a descriptor list (one descriptor per distinct source block): HBM-tier
+// sources go to `desc`, host-tier sources to `desc_host`, so that each tier gets the copy engine and the grid
+// that suit it (HBM bandwidth needs every SM, the host link is saturated by a few CTAs)
 __global__ void __launch_bounds__(256) fetch_link_kernel(Store st, const int* __restrict__ ids, const int* __restrict__ matched,
                                                          const int* __restrict__ bt, int R, int max_blocks, u32 cache_blocks,
-                                                         u32* __restrict__ head, int2* __restrict__ node, int2* __restrict__ desc) {
+                                                         u32* __restrict__ head, int2* __restrict__ node, int2* __restrict__ desc,
+                                                         int2* __restrict__ desc_host) {
   const long long total = (long long)R * max_blocks;
   const long long rounded = (total + 31) & ~31ll;
   const int lane = threadIdx.x & 31;
@@ -524,16 +527,22 @@ __global__ void __launch_bounds__(256) fetch_link_kernel(Store st, const int* __
         }
       }
     }
-    const unsigned m = __ballot_sync(FULL, first);
+    const bool on_host = first && (u32)id >= st.n[0];
+    const unsigned m = __ballot_sync(FULL, first && !on_host);
+    const unsigned mh = __ballot_sync(FULL, on_host);
     if (m) {
       u32 base = 0;
-      if (lane == __ffs(m) - 1) {
-        base = atomicAdd(&st.ctrl->n_pairs, (u32)__popc(m));
-        atomicAdd(&st.ctrl->blocks_fetched_distinct, (u64)__popc(m));
-      }
+      if (lane == __ffs(m) - 1) base = atomicAdd(&st.ctrl->n_pairs, (u32)__popc(m));
       base = __shfl_sync(FULL, base, __ffs(m) - 1);
-      if (first) desc[base + __popc(m & ((1u << lane) - 1u))] = make_int2(id, 0);
+      if (first && !on_host) desc[base + __popc(m & ((1u << lane) - 1u))] = make_int2(id, 0);
     }
+    if (mh) {
+      u32 base = 0;
+      if (lane == __ffs(mh) - 1) base = atomicAdd(&st.ctrl->n_pairs_host, (u32)__popc(mh));
+      base = __shfl_sync(FULL, base, __ffs(mh) - 1);
+      if (on_host) desc_host[base + __popc(mh & ((1u << lane) - 1u))] = make_int2(id, 0);
+    }
+    if ((m | mh) && lane == 0) atomicAdd(&st.ctrl->blocks_fetched_distinct, (u64)(__popc(m) + __popc(mh)));
   }
   cnt0 = __reduce_add_sync(FULL, cnt0);
   cnt1 = __reduce_add_sync(FULL, cnt1);

@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(256) demote_finish_kernel(Store st, const Key2
     c->ring[0].count += take;
     c->live[0] -= take;
     c->live[1] += take;
-    c->n_pairs = take;
+    c->n_pairs_tier = take;
     c->blocks_demoted += take;
     if (st.policy && take && sorted[take - 1].hi > c->inflation) c->inflation = sorted[take - 1].hi;
     if (n_evicted) { n_evicted[0] = (int)take; n_evicted[1] = (int)dropped; }

@@ -23,7 +23,7 @@ inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
   u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
-      cta_sums, prefix, promo_first, promo_cnt, links, total;
+      cta_sums, prefix, promo_first, promo_cnt, links, desc_tier, desc_host, total;
   u32 n_tiles;
 };
 
@@ -63,6 +63,8 @@ Layout make_layout(const ptstore_config_t* c) {
   L.promo_first = take(N * 4);
   L.promo_cnt = take(N * 4);
   L.links = take(M * sizeof(int2));
+  L.desc_tier = take((u64)c->hbm_blocks * sizeof(int2));
+  L.desc_host = take((c->host_blocks ? (M < c->host_blocks ? M : (u64)c->host_blocks) : 1) * sizeof(int2));
   L.total = o;
   return L;
 }
@@ -88,6 +90,12 @@ struct ptstore {
   u32* promo_first;
   u32* promo_cnt;
   int2* links;           // fetch: destination list nodes, one per (request, block) entry
+  int2* desc_tier;       // demotion: {HBM id, host id} pairs
+  int2* desc_host;       // fetch: descriptors of distinct host-tier source blocks
+  int host_ctas;         // grid of the copies that run at host-link speed
+  cudaStream_t tier_stream;   // side stream of ptstore_evict_async (created on first use)
+  cudaEvent_t ev_meta, ev_copy;
+  bool tier_ready, tier_pending;
   u64 epoch;
   u64 launches;
   int last_cuda;
@@ -248,7 +256,14 @@ int launch_bulk_multi(ptstore* h, const Paged& pc, cudaStream_t s, BulkVariant v
 }
 
 template <int MODE>
-int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream_t s) {
+int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream_t s, const int2* desc = nullptr,
+                const u32* n_pairs = nullptr, int grid = 0) {
+  if (!desc) { desc = h->desc; n_pairs = &h->st.ctrl->n_pairs; }
+  if (grid > 0) {       // host-link copies: fixed small grid, vector engine
+    copy_vector_kernel<MODE, 256, 8><<<grid, 256, 0, s>>>(h->st, pc, desc, n_pairs);
+    PTS_CHECK_LAUNCH(h);
+    return PTSTORE_OK;
+  }
   const u32 variant = (h->cfg.flags >> 16) & 0xFu;
   int per_sm = (int)((h->cfg.flags >> 20) & 0xFFu);
   if ((h->cfg.flags & PTSTORE_COPY_BULK) && !host_side_possible) {
@@ -260,13 +275,13 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
   }
   switch (variant) {
     case 1:
-      copy_vector_kernel<MODE, 256, 8><<<h->sms * (per_sm ? per_sm : 8), 256, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
+      copy_vector_kernel<MODE, 256, 8><<<h->sms * (per_sm ? per_sm : 8), 256, 0, s>>>(h->st, pc, desc, n_pairs);
       break;
     case 2:
-      copy_vector_kernel<MODE, 512, 4><<<h->sms * (per_sm ? per_sm : 4), 512, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
+      copy_vector_kernel<MODE, 512, 4><<<h->sms * (per_sm ? per_sm : 4), 512, 0, s>>>(h->st, pc, desc, n_pairs);
       break;
     default:
-      copy_vector_kernel<MODE, 256, 4><<<h->sms * (per_sm ? per_sm : 16), 256, 0, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs);
+      copy_vector_kernel<MODE, 256, 4><<<h->sms * (per_sm ? per_sm : 16), 256, 0, s>>>(h->st, pc, desc, n_pairs);
       break;
   }
   PTS_CHECK_LAUNCH(h);
@@ -348,6 +363,59 @@ int run_drop(ptstore* h, int tier, int mode, u32 n, int* n_evicted, int* victims
   return PTSTORE_OK;
 }
 
+// make `s` wait for a demotion copy that ptstore_evict_async left running on the side stream
+int join_tier(ptstore* h, cudaStream_t s) {
+  if (!h->tier_pending) return PTSTORE_OK;
+  if (cudaStreamWaitEvent(s, h->ev_copy, 0) != cudaSuccess) { h->last_cuda = (int)cudaGetLastError(); return PTSTORE_E_CUDA; }
+  h->tier_pending = false;
+  return PTSTORE_OK;
+}
+
+int evict_impl(ptstore* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, cudaStream_t s, bool async_copy) {
+  if (!h || n_blocks < 0 || (tier != PTSTORE_TIER_HBM && tier != PTSTORE_TIER_HOST) || !n_evicted) return PTSTORE_E_INVAL;
+  if (tier == PTSTORE_TIER_HOST && h->cfg.host_blocks == 0) return PTSTORE_E_INVAL;
+  int rc = join_tier(h, s);
+  if (rc) return rc;
+  const u32 n = (u32)n_blocks;
+  if (tier == PTSTORE_TIER_HOST || h->cfg.host_blocks == 0) return run_drop(h, tier, EV_DROP, n, n_evicted, victim_ids, s);
+  // HBM tier with a host tier behind it: make room in the host ring, then demote
+  rc = run_drop(h, 1, EV_HOST_ROOM, n, nullptr, nullptr, s);
+  if (rc) return rc;
+  const int cap = h->sms * 8;
+  evict_begin_kernel<<<1, 1, 0, s>>>(h->st, EV_DEMOTE, n);
+  PTS_CHECK_LAUNCH(h);
+  collect_kernel<<<grid_for(h->cfg.hbm_blocks, 256, cap), 256, 0, s>>>(h->st, 0, nullptr, h->sort_buf[0]);
+  PTS_CHECK_LAUNCH(h);
+  int res;
+  rc = launch_sort(h, s, &res);
+  if (rc) return rc;
+  apply_demote_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, h->sort_buf[res], h->desc_tier, victim_ids);
+  PTS_CHECK_LAUNCH(h);
+  demote_finish_kernel<<<1, 256, 0, s>>>(h->st, h->sort_buf[res], n_evicted, victim_ids, h->room);
+  PTS_CHECK_LAUNCH(h);
+  Paged none = {};
+  if (!async_copy) return launch_copy<COPY_POOL>(h, none, true, s, h->desc_tier, &h->st.ctrl->n_pairs_tier, h->host_ctas);
+  // the copy HBM -> host goes to the side stream, ordered after the metadata kernels above
+  if (!h->tier_ready) {
+    if (cudaStreamCreateWithFlags(&h->tier_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_meta, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_copy, cudaEventDisableTiming) != cudaSuccess) {
+      h->last_cuda = (int)cudaGetLastError();
+      return PTSTORE_E_CUDA;
+    }
+    h->tier_ready = true;
+  }
+  if (cudaEventRecord(h->ev_meta, s) != cudaSuccess || cudaStreamWaitEvent(h->tier_stream, h->ev_meta, 0) != cudaSuccess) {
+    h->last_cuda = (int)cudaGetLastError();
+    return PTSTORE_E_CUDA;
+  }
+  rc = launch_copy<COPY_POOL>(h, none, true, h->tier_stream, h->desc_tier, &h->st.ctrl->n_pairs_tier, h->host_ctas);
+  if (rc) return rc;
+  if (cudaEventRecord(h->ev_copy, h->tier_stream) != cudaSuccess) { h->last_cuda = (int)cudaGetLastError(); return PTSTORE_E_CUDA; }
+  h->tier_pending = true;
+  return PTSTORE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -413,6 +481,14 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->promo_first = reinterpret_cast<u32*>(w + lay.promo_first);
   h->promo_cnt = reinterpret_cast<u32*>(w + lay.promo_cnt);
   h->links = reinterpret_cast<int2*>(w + lay.links);
+  h->desc_tier = reinterpret_cast<int2*>(w + lay.desc_tier);
+  h->desc_host = reinterpret_cast<int2*>(w + lay.desc_host);
+  {
+    // a few CTAs saturate the host link; keeping these grids small leaves the SMs to kernels that run beside them
+    const char* e = std::getenv("PTSTORE_HOST_CTAS");
+    const int v = e ? std::atoi(e) : 0;
+    h->host_ctas = v > 0 ? v : 32;
+  }
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int cap = sms * 8;
@@ -430,6 +506,12 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
 
 int ptstore_destroy(ptstore_t* h) {
   if (!h) return PTSTORE_E_INVAL;
+  if (h->tier_ready) {
+    cudaStreamSynchronize(h->tier_stream);
+    cudaEventDestroy(h->ev_meta);
+    cudaEventDestroy(h->ev_copy);
+    cudaStreamDestroy(h->tier_stream);
+  }
   delete h;
   return PTSTORE_OK;
 }
@@ -481,12 +563,14 @@ int ptstore_fetch(ptstore_t* h, const int32_t* block_ids, const int32_t* matched
   fetch_begin_kernel<<<grid_for(n_blocks, 256, cap), 256, 0, s>>>(h->st, h->promo_first, n_blocks);
   PTS_CHECK_LAUNCH(h);
   fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, block_tables, R, max_blocks,
-                                                                                 dst->num_blocks, h->promo_first, h->links, h->desc);
+                                                                                 dst->num_blocks, h->promo_first, h->links, h->desc, h->desc_host);
   PTS_CHECK_LAUNCH(h);
   Paged pc = to_paged(dst);
   pc.head = h->promo_first;
   pc.node = h->links;
-  return launch_copy<COPY_FETCH_MULTI>(h, pc, h->cfg.host_blocks > 0, s);
+  rc = launch_copy<COPY_FETCH_MULTI>(h, pc, false, s);                    // HBM-tier sources: every SM
+  if (rc || h->cfg.host_blocks == 0) return rc;
+  return launch_copy<COPY_FETCH_MULTI>(h, pc, true, s, h->desc_host, &h->st.ctrl->n_pairs_host, h->host_ctas);   // host-tier sources
 }
 
 int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
@@ -504,6 +588,8 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   h->epoch += 1;
   if (R == 0) return PTSTORE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rc = join_tier(h, s);        // new blocks may reuse HBM ids whose demotion copy is still running
+  if (rc) return rc;
   rc = maybe_rebuild(h, s);
   if (rc) return rc;
   const long long* off = reinterpret_cast<const long long*>(offsets);
@@ -545,28 +631,16 @@ int ptstore_release(ptstore_t* h, const int32_t* block_ids, const int32_t* match
 }
 
 int ptstore_evict(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, ptstore_stream_t stream) {
-  if (!h || n_blocks < 0 || (tier != PTSTORE_TIER_HBM && tier != PTSTORE_TIER_HOST) || !n_evicted) return PTSTORE_E_INVAL;
-  if (tier == PTSTORE_TIER_HOST && h->cfg.host_blocks == 0) return PTSTORE_E_INVAL;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const u32 n = (u32)n_blocks;
-  if (tier == PTSTORE_TIER_HOST || h->cfg.host_blocks == 0) return run_drop(h, tier, EV_DROP, n, n_evicted, victim_ids, s);
-  // HBM tier with a host tier behind it: make room in the host ring, then demote
-  int rc = run_drop(h, 1, EV_HOST_ROOM, n, nullptr, nullptr, s);
-  if (rc) return rc;
-  const int cap = h->sms * 8;
-  evict_begin_kernel<<<1, 1, 0, s>>>(h->st, EV_DEMOTE, n);
-  PTS_CHECK_LAUNCH(h);
-  collect_kernel<<<grid_for(h->cfg.hbm_blocks, 256, cap), 256, 0, s>>>(h->st, 0, nullptr, h->sort_buf[0]);
-  PTS_CHECK_LAUNCH(h);
-  int res;
-  rc = launch_sort(h, s, &res);
-  if (rc) return rc;
-  apply_demote_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, h->sort_buf[res], h->desc, victim_ids);
-  PTS_CHECK_LAUNCH(h);
-  demote_finish_kernel<<<1, 256, 0, s>>>(h->st, h->sort_buf[res], n_evicted, victim_ids, h->room);
-  PTS_CHECK_LAUNCH(h);
-  Paged none = {};
-  return launch_copy<COPY_POOL>(h, none, true, s);
+  return evict_impl(h, tier, n_blocks, n_evicted, victim_ids, static_cast<cudaStream_t>(stream), false);
+}
+
+int ptstore_evict_async(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, ptstore_stream_t stream) {
+  return evict_impl(h, tier, n_blocks, n_evicted, victim_ids, static_cast<cudaStream_t>(stream), true);
+}
+
+int ptstore_join(ptstore_t* h, ptstore_stream_t stream) {
+  if (!h) return PTSTORE_E_INVAL;
+  return join_tier(h, static_cast<cudaStream_t>(stream));
 }
 
 int ptstore_promote(ptstore_t* h, int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks, uint32_t flags,
@@ -576,6 +650,8 @@ int ptstore_promote(ptstore_t* h, int32_t* block_ids, const int32_t* matched_blo
   if (h->cfg.host_blocks == 0 || max_promote < 0) return PTSTORE_E_INVAL;
   if (R > 0 && (!block_ids || !matched_blocks)) return PTSTORE_E_INVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rc = join_tier(h, s);
+  if (rc) return rc;
   const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
   if (cudaMemsetAsync(h->promo_first, 0xFF, N * 4, s) != cudaSuccess || cudaMemsetAsync(h->promo_cnt, 0, N * 4, s) != cudaSuccess) {
     h->last_cuda = (int)cudaGetLastError();
@@ -601,7 +677,7 @@ int ptstore_promote(ptstore_t* h, int32_t* block_ids, const int32_t* matched_blo
   promote_rewrite_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first);
   PTS_CHECK_LAUNCH(h);
   Paged none = {};
-  return launch_copy<COPY_POOL>(h, none, true, s);
+  return launch_copy<COPY_POOL>(h, none, true, s, nullptr, nullptr, h->host_ctas);      // host -> HBM at host-link speed
 }
 
 int ptstore_status(ptstore_t* h, ptstore_stream_t stream, uint32_t* status_out) {

@@ -84,9 +84,9 @@ class Pair:
         self.o.release(ids, matched)
         self.g.release(dev(ids), dev(matched))
 
-    def evict(self, tier, n, literal=True):
+    def evict(self, tier, n, literal=True, asynchronous=False):
         ne_o, v_o = self.o.evict(tier, n, literal=literal)
-        ne_g, v_g = self.g.evict(tier, n)
+        ne_g, v_g = self.g.evict(tier, n, asynchronous=asynchronous)
         ne_g = ne_g.cpu().numpy()
         assert ne_o.tolist() == ne_g.tolist(), ("evicted counts differ", ne_o, ne_g)
         k = int(ne_o.sum())
@@ -100,6 +100,8 @@ class Pair:
 
     def check_pools(self):
         """Every live block's bytes agree (free blocks may hold stale data on either side)."""
+        self.g.join()
+        torch.cuda.synchronize()
         pool_g = self.g.hbm_pool.cpu().numpy().reshape(self.g.hbm_blocks, -1)
         pool_o = self.o.pool(0)
         host_g = self.g.host_pool.numpy().reshape(self.g.host_blocks, -1) if self.g.host_blocks else None

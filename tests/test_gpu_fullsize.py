@@ -116,7 +116,7 @@ def test_churn_with_host_tier():
     demoted = dropped = promoted = 0
     for k in range(n_steps):
         seqs, tags = st.batch(16)
-        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9), promote=(256 if k >= 30 else 0))
+        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9), promote=(256 if k >= 30 else 0), async_demote=(k >= 20 and k % 2 == 0))
         promoted += r["promoted"]
         if r["evicted"] is not None:
             demoted += int(r["evicted"][0]); dropped += int(r["evicted"][1])

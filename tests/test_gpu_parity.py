@@ -124,8 +124,9 @@ def test_insert_dedupe_denial_and_alloc_order():
     p.close()
 
 
-@pytest.mark.parametrize("host,policy", [(0, "lru"), (24, "lru"), (0, "gdsf"), (24, "gdsf")])
-def test_random_churn_lockstep(host, policy):
+@pytest.mark.parametrize("host,policy,async_demote", [(0, "lru", False), (24, "lru", False), (0, "gdsf", False), (24, "gdsf", False),
+                                                      (24, "lru", True)])
+def test_random_churn_lockstep(host, policy, async_demote):
     """Random interleaving of lookup(PIN) / fetch / evict / insert / release, compared call by call."""
     Pair, dev, G = _imports()
     sh = W.KVShape(2, 1, 8, 2)
@@ -154,10 +155,13 @@ def test_random_churn_lockstep(host, policy):
                     bt[r, j] = perm[k]; k += 1
             if host and rng.random() < 0.6:                    # move some of the host-tier hits into HBM first
                 io, _n = p.promote(io, mo, True, int(rng.integers(0, 6)))
+            tier = int(rng.integers(0, 2)) if host else 0
+            n_ev = int(rng.integers(0, 12))
+            if async_demote and op < 0.7:                      # demotion copy on the side stream, overlapping the fetch
+                p.evict(tier, n_ev, literal=bool(step % 2), asynchronous=True)
             p.fetch(io, mo, dst, bt)
-            if op < 0.7:
-                tier = int(rng.integers(0, 2)) if host else 0
-                p.evict(tier, int(rng.integers(0, 12)), literal=bool(step % 2))
+            if not async_demote and op < 0.7:
+                p.evict(tier, n_ev, literal=bool(step % 2))
             need = sum(len(x) // B for x in batch)
             src = W.random_kv_cache(seed * 1000 + step, sh, need + 1)
             sbt = W.shuffled_block_tables(rng, batch, B, mb, need + 1)
