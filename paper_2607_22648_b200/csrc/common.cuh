@@ -170,6 +170,51 @@ __device__ __forceinline__ u32 find_slot(const Slot* __restrict__ table, u64 slo
   return NO_SLOT;
 }
 
+// The same probe in two halves, so that a caller can put independent work between the loads of the first window and
+// their use: probe_issue starts the loads, probe_finish examines them and walks on if the run is longer.
+struct ProbeWindow { uint4 v[PROBE_WINDOW]; };
+__device__ __forceinline__ void probe_issue(const Slot* __restrict__ table, u64 slots, u64 key, ProbeWindow& w) {
+  const u64 s = home_slot(key, slots);
+#pragma unroll
+  for (int k = 0; k < PROBE_WINDOW; ++k) {
+    u64 t = s + k;
+    t = t >= slots ? t - slots : t;
+    w.v[k] = *reinterpret_cast<const uint4*>(table + t);
+  }
+}
+__device__ __forceinline__ u32 probe_finish(const Slot* __restrict__ table, u64 slots, u64 key, const ProbeWindow& w, u32* visited) {
+  u32 n = 0;
+#pragma unroll
+  for (int k = 0; k < PROBE_WINDOW; ++k) {
+    const u64 kk = ((u64)w.v[k].y << 32) | w.v[k].x;
+    ++n;
+    if (kk == key) { *visited = n; return w.v[k].z; }
+    if (kk == KEY_EMPTY) { *visited = n; return NO_ID; }
+  }
+  u64 s = home_slot(key, slots) + PROBE_WINDOW;
+  if (s >= slots) s -= slots;
+  for (u64 i = PROBE_WINDOW; i < slots; i += PROBE_WINDOW) {
+    uint4 v[PROBE_WINDOW];
+#pragma unroll
+    for (int k = 0; k < PROBE_WINDOW; ++k) {
+      u64 t = s + k;
+      t = t >= slots ? t - slots : t;
+      v[k] = *reinterpret_cast<const uint4*>(table + t);
+    }
+#pragma unroll
+    for (int k = 0; k < PROBE_WINDOW; ++k) {
+      const u64 kk = ((u64)v[k].y << 32) | v[k].x;
+      ++n;
+      if (kk == key) { *visited = n; return v[k].z; }
+      if (kk == KEY_EMPTY) { *visited = n; return NO_ID; }
+    }
+    s += PROBE_WINDOW;
+    if (s >= slots) s -= slots;
+  }
+  *visited = n;
+  return NO_ID;
+}
+
 __device__ __forceinline__ int tier_of(const Store& st, u32 id) { return id < st.n[0] ? 0 : 1; }
 __device__ __forceinline__ unsigned char* block_ptr(const Store& st, u32 id) {
   return id < st.n[0] ? st.pool[0] + (u64)id * st.block_bytes : st.pool[1] + (u64)(id - st.n[0]) * st.block_bytes;

@@ -18,10 +18,14 @@ template <int L>
 __device__ __forceinline__ u64 chain_chunk(u64& parent, u64 c, int lane, int steps) {
   const int sl = lane & (L - 1), base_lane = lane & ~(L - 1);
   u64 k = parent, mine = 0;
+  // the chain itself is serial (three dependent 64-bit multiplies per step); the shuffle that brings the next
+  // block's content hash is issued one step ahead so that its latency hides behind the arithmetic
+  u64 ci = __shfl_sync(FULL, c, base_lane);
   for (int i = 0; i < steps; ++i) {
-    u64 ci = __shfl_sync(FULL, c, base_lane + i);
+    const u64 cn = __shfl_sync(FULL, c, base_lane + ((i + 1) & (L - 1)));
     k = hchain(k, ci);
     if (sl == i) mine = k;
+    ci = cn;
   }
   return mine;
 }
@@ -134,6 +138,118 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
   my_visited = __reduce_add_sync(FULL, my_visited);
   if (lane < 4) {
     const u32 v = lane == 0 ? qb : lane == 1 ? my_probes : lane == 2 ? my_visited : mb;
+    if (v) atomicAdd(&st.ctrl->lookup_stripes[warp % LOOKUP_STRIPES][lane], (u64)v);
+  }
+}
+
+// ---- split path for few, long requests ---------------------------------------------------------------------------
+// With a whole warp per request the fused kernel above is one dependent chain per 32-block chunk: token loads ->
+// content hashes -> 32 chain steps -> probe.  For long prompts (hundreds of blocks, a handful of requests) that
+// serial latency is all there is.  Here the content hashes of ALL blocks are computed first by one thread per block
+// (content_kernel), and the per-request warp only chains and probes; the probe loads of a chunk are in flight while
+// the keys of the next chunk are chained (the chain does not depend on the probe result; if the chunk then turns out
+// to hold the first miss the extra chain is discarded).
+__global__ void __launch_bounds__(256) content_kernel(Store st, const int* __restrict__ tokens, const long long* __restrict__ offsets,
+                                                      int R, int max_blocks, u64* __restrict__ content_out) {
+  const long long total = (long long)R * max_blocks;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
+    if (j >= full_blocks(offsets, r, st.block_tokens, max_blocks)) continue;
+    content_out[e] = content_block(tokens + offsets[r] + (long long)j * st.block_tokens, st.block_tokens);
+  }
+}
+
+// keys[r][j] = chained key from content[r][j]; may run in place (content == keys)
+__global__ void __launch_bounds__(128) chain_kernel(Store st, const u64* content, const long long* __restrict__ offsets, int R,
+                                                    int max_blocks, u64* keys_out) {
+  const int lane = threadIdx.x & 31;
+  const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (r >= R) return;
+  const int nblk = full_blocks(offsets, (int)r, st.block_tokens, max_blocks);
+  u64 parent = st.root_key;
+  u64 c_next = lane < nblk ? content[r * max_blocks + lane] : 0;          // loaded a chunk ahead of its use
+  for (int base = 0; base < nblk; base += 32) {
+    const int j = base + lane;
+    const u64 c = c_next;
+    c_next = j + 32 < nblk ? content[r * max_blocks + j + 32] : 0;
+    const int steps = nblk - base < 32 ? nblk - base : 32;
+    const u64 key = chain_chunk<32>(parent, c, lane, steps);
+    if (j < nblk) keys_out[r * max_blocks + j] = key;
+    parent = __shfl_sync(FULL, key, 31);
+  }
+  for (int j = nblk + lane; j < max_blocks; j += 32) keys_out[r * max_blocks + j] = 0;
+}
+
+__global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* __restrict__ content, const long long* __restrict__ offsets,
+                                                           int R, int max_blocks, u32 flags, u64 epoch, int* __restrict__ matched,
+                                                           int* __restrict__ ids_out) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long r = warp;
+  if (r >= R) return;
+  const int nblk = full_blocks(offsets, (int)r, st.block_tokens, max_blocks);
+  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
+  const u64* crow = content + r * max_blocks;
+  int m = 0;
+  u32 probes = 0, visited_sum = 0;
+  u64 parent = st.root_key;
+  u64 key = 0;
+  u64 c_next = 0;                                  // content hashes of the chunk after the current one, loaded a chunk ahead
+  if (nblk > 0) {
+    const u64 c0 = lane < nblk ? crow[lane] : 0;
+    c_next = 32 + lane < nblk ? crow[32 + lane] : 0;
+    key = chain_chunk<32>(parent, c0, lane, nblk < 32 ? nblk : 32);
+  }
+  for (int base = 0; base < nblk; base += 32) {
+    const int j = base + lane;
+    const bool active = j < nblk;
+    ProbeWindow w;
+    if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
+    u64 next_key = 0;
+    if (base + 32 < nblk) {                                       // ... while the next chunk is chained
+      const u64 cn = c_next;
+      c_next = base + 64 + lane < nblk ? crow[base + 64 + lane] : 0;
+      u64 p = __shfl_sync(FULL, key, 31);
+      const int left = nblk - base - 32;
+      next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
+    }
+    u32 id = NO_ID;
+    if (active) {
+      u32 visited;
+      id = probe_finish(st.table, st.slots, key, w, &visited);
+      probes += 1;
+      visited_sum += visited;
+    }
+    const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
+    const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);
+    const bool hit = active && lane < nf;
+    const unsigned hm = __ballot_sync(FULL, hit);
+    if (hit) {
+      ids_out[r * max_blocks + j] = (int)id;
+      const bool touch = !(flags & F_NO_TOUCH);
+      if (touch && st.policy == 0) st.m_last[id] = epoch;
+      if ((flags & F_PIN) || (touch && st.policy)) {
+        const unsigned same = __match_any_sync(hm, id);            // ids of one request are distinct: groups of one
+        if (lane == __ffs(same) - 1) {
+          const u32 cnt = (u32)__popc(same);
+          if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
+          if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
+        }
+      }
+    }
+    m += nf;
+    if (nf < 32) break;
+    key = next_key;
+  }
+  for (int j = m + lane; j < max_blocks; j += 32) ids_out[r * max_blocks + j] = -1;
+  if (lane == 0) matched[r] = m;
+  u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
+  probes = __reduce_add_sync(FULL, probes);
+  visited_sum = __reduce_add_sync(FULL, visited_sum);
+  qb = __reduce_add_sync(FULL, qb);
+  mb = __reduce_add_sync(FULL, mb);
+  if (lane < 4) {
+    const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
     if (v) atomicAdd(&st.ctrl->lookup_stripes[warp % LOOKUP_STRIPES][lane], (u64)v);
   }
 }

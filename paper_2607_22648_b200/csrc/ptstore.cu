@@ -167,6 +167,26 @@ int launch_lookup(ptstore* h, const int* tokens, const long long* offsets, int R
 // Lanes per request.  Many requests: narrow sub-warps (fewer blocks hashed and probed past the first miss,
 // 32/L requests per warp).  Few long requests: a whole warp per request (fewer serial chunks).
 // Measured on the 16,384 x 64-block lookup stress: L=8 33 us, L=16 37 us, L=32 63 us per call.
+// few long requests: content hashes by one thread per block, then one warp per request chains and probes
+bool split_path(const ptstore* h, int R, int max_blocks) {
+  const u32 forced = (h->cfg.flags >> 8) & 0xFFu;
+  return forced == 0 && R < 1024 && max_blocks > 32;
+}
+
+int launch_content(ptstore* h, const int* tokens, const long long* offsets, int R, int max_blocks, u64* out, cudaStream_t s) {
+  content_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, tokens, offsets, R, max_blocks, out);
+  PTS_CHECK_LAUNCH(h);
+  return PTSTORE_OK;
+}
+
+int launch_hash_split(ptstore* h, const int* tokens, const long long* offsets, int R, int max_blocks, u64* keys, cudaStream_t s) {
+  int rc = launch_content(h, tokens, offsets, R, max_blocks, keys, s);
+  if (rc) return rc;
+  chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, keys, offsets, R, max_blocks, keys);       // in place
+  PTS_CHECK_LAUNCH(h);
+  return PTSTORE_OK;
+}
+
 int lanes_for(const ptstore* h, int R, int max_blocks) {
   const u32 forced = (h->cfg.flags >> 8) & 0xFFu;
   if (forced == 8 || forced == 16 || forced == 32) return (int)forced;
@@ -525,6 +545,7 @@ int ptstore_hash(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, in
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const long long* off = reinterpret_cast<const long long*>(offsets);
   u64* ko = reinterpret_cast<u64*>(keys_out);
+  if (split_path(h, R, max_blocks)) return launch_hash_split(h, tokens, off, R, max_blocks, ko, s);
   switch (lanes_for(h, R, max_blocks)) {
     case 8: return launch_hash<8>(h, tokens, off, R, max_blocks, ko, s);
     case 16: return launch_hash<16>(h, tokens, off, R, max_blocks, ko, s);
@@ -541,6 +562,13 @@ int ptstore_lookup(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   if (R == 0) return PTSTORE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const long long* off = reinterpret_cast<const long long*>(offsets);
+  if (split_path(h, R, max_blocks)) {
+    rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
+    if (rc) return rc;
+    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids);
+    PTS_CHECK_LAUNCH(h);
+    return PTSTORE_OK;
+  }
   switch (lanes_for(h, R, max_blocks)) {
     case 8: return launch_lookup<8>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
     case 16: return launch_lookup<16>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
@@ -593,7 +621,8 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   rc = maybe_rebuild(h, s);
   if (rc) return rc;
   const long long* off = reinterpret_cast<const long long*>(offsets);
-  switch (lanes_for(h, R, max_blocks)) {
+  if (split_path(h, R, max_blocks)) rc = launch_hash_split(h, tokens, off, R, max_blocks, h->keys, s);
+  else switch (lanes_for(h, R, max_blocks)) {
     case 8: rc = launch_hash<8>(h, tokens, off, R, max_blocks, h->keys, s); break;
     case 16: rc = launch_hash<16>(h, tokens, off, R, max_blocks, h->keys, s); break;
     default: rc = launch_hash<32>(h, tokens, off, R, max_blocks, h->keys, s); break;
