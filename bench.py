@@ -193,6 +193,8 @@ class Serving:
         self.h_matched = torch.empty(R, dtype=torch.int32).pin_memory()
         self.h_ids = torch.empty((R, self.mb), dtype=torch.int32).pin_memory()
         self.h_newb = torch.empty(R, dtype=torch.int32).pin_memory()
+        self.h_stats = torch.zeros(ctypes_sizeof_stats(self.G), dtype=torch.uint8).pin_memory()
+        self.after_lookup = torch.cuda.Event()
 
     def step(self, i, e2e=False, events=None):
         """One pass of the path.  Returns nothing; counters come from ptstore_stats."""
@@ -209,6 +211,9 @@ class Serving:
             st.promote(self.ids, self.matched, G.PINNED_LIST, self.promote, self.nprom)
             if events is not None:
                 events["promote"][-1] = (events["promote"][-1][0], self._ev())
+        self.h_matched.copy_(self.matched, non_blocking=True)
+        st.stats_enqueue(self.h_stats)
+        self.after_lookup.record()
         if self.async_demote:
             self._evict_shortfall(s, events)          # its demotion copy (device -> host) overlaps the fetch (host -> device)
         if events is not None:
@@ -229,10 +234,11 @@ class Serving:
             self.h_newb.copy_(self.newb, non_blocking=True)
 
     def _evict_shortfall(self, s, events):
-        # the serving engine needs the matched lengths on the host anyway; the same sync gives the free count
+        # the serving engine needs the matched lengths on the host anyway; the counters come back with them, behind an event
+        # recorded right after the lookup, so the host does not wait for the fetch that is already queued
         torch, G, st = self.torch, self.G, self.store
-        self.h_matched.copy_(self.matched, non_blocking=True)
-        stats = st.stats()
+        self.after_lookup.synchronize()
+        stats = G.Stats.from_buffer_copy(self.h_stats.numpy().tobytes())
         need = s["total_blocks"] - int(self.h_matched.sum()) + self.promote      # keep room for the next step's promotions
         short = need - int(stats.free_blocks[0])
         if short > 0:
@@ -252,6 +258,11 @@ class Serving:
         h2d = sum(v.numel() * v.element_size() for v in s["host"].values())
         d2h = self.h_matched.numel() * 4 + self.h_ids.numel() * 4 + self.h_newb.numel() * 4
         return h2d, d2h
+
+
+def ctypes_sizeof_stats(G):
+    import ctypes
+    return ctypes.sizeof(G.Stats)
 
 
 def reduce_over_ranks(dist, x, op, device):

@@ -269,6 +269,14 @@ int ptstore_status(ptstore_t* st, ptstore_stream_t stream, uint32_t* status_out 
 /* Synchronise `stream` and copy the counters to *out (host). */
 int ptstore_stats(ptstore_t* st, ptstore_stream_t stream, ptstore_stats_t* out /*host*/);
 
+/*
+ * The same counters without blocking: a one-thread kernel on `stream` writes them to *out, which must be
+ * device-accessible (device memory, or pinned host memory the device can write).  The caller waits for the stream,
+ * or for an event recorded after this call, before reading.  Lets a scheduler learn the free-block count behind a
+ * lookup while the fetch that follows is already running.
+ */
+int ptstore_stats_enqueue(ptstore_t* st, ptstore_stats_t* out /*device-accessible*/, ptstore_stream_t stream);
+
 /* Number of this library's kernels launched through the handle so far (host counter, no sync). */
 uint64_t ptstore_launch_count(const ptstore_t* st);
 

@@ -57,7 +57,7 @@ class Stats(C.Structure):
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
-           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join"]
+           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join", "ptstore_stats_enqueue"]
 
 
 def _load():
@@ -81,6 +81,7 @@ def _load():
     lib.ptstore_promote.argtypes = [vp, vp, vp, i32, i32, u32, i32, vp, vp]
     lib.ptstore_status.argtypes = [vp, vp, C.POINTER(u32)]
     lib.ptstore_stats.argtypes = [vp, vp, C.POINTER(Stats)]
+    lib.ptstore_stats_enqueue.argtypes = [vp, vp, vp]
     lib.ptstore_launch_count.restype = u64
     lib.ptstore_launch_count.argtypes = [vp]
     lib.ptstore_last_cuda_error.argtypes = [vp]
@@ -258,6 +259,11 @@ class PTStore:
         out = Stats()
         self._check(lib.ptstore_stats(self.h, _stream(), C.byref(out)), "ptstore_stats")
         return out
+
+    def stats_enqueue(self, pinned_bytes):
+        """Writes the counters into `pinned_bytes` (a pinned uint8 host tensor of sizeof(Stats)) without blocking;
+        read it with Stats.from_buffer_copy(...) once the stream (or a later event) has completed."""
+        self._check(lib.ptstore_stats_enqueue(self.h, pinned_bytes.data_ptr(), _stream()), "ptstore_stats_enqueue")
 
     def launch_count(self):
         return int(lib.ptstore_launch_count(self.h))

@@ -303,4 +303,29 @@ __global__ void ctrl_init_kernel(Store st) {
   c->ring[1].count = st.n[1];
 }
 
+// counters for a caller that does not want to block: written by the device to any device-accessible address
+struct StatsOut {
+  u64 epoch, live[2], free_blocks[2], tombstones, query_blocks, probes_issued, slots_visited, blocks_matched, blocks_fetched[2],
+      blocks_inserted, blocks_denied, blocks_dropped[2], blocks_demoted, rebuilds, blocks_promoted, gdsf_clock, blocks_fetched_distinct;
+};
+__global__ void stats_kernel(Store st, u64 epoch, StatsOut* __restrict__ out) {
+  const Ctrl* c = st.ctrl;
+  StatsOut o;
+  o.epoch = epoch;
+  for (int t = 0; t < 2; ++t) {
+    o.live[t] = c->live[t]; o.free_blocks[t] = c->ring[t].count;
+    o.blocks_fetched[t] = c->blocks_fetched[t]; o.blocks_dropped[t] = c->blocks_dropped[t];
+  }
+  o.tombstones = c->tombstones;
+  o.query_blocks = c->query_blocks; o.probes_issued = c->probes_issued; o.slots_visited = c->slots_visited; o.blocks_matched = c->blocks_matched;
+  for (int i = 0; i < LOOKUP_STRIPES; ++i) {
+    o.query_blocks += c->lookup_stripes[i][0]; o.probes_issued += c->lookup_stripes[i][1];
+    o.slots_visited += c->lookup_stripes[i][2]; o.blocks_matched += c->lookup_stripes[i][3];
+  }
+  o.blocks_inserted = c->blocks_inserted; o.blocks_denied = c->blocks_denied; o.blocks_demoted = c->blocks_demoted;
+  o.rebuilds = c->rebuilds; o.blocks_promoted = c->blocks_promoted; o.gdsf_clock = c->inflation;
+  o.blocks_fetched_distinct = c->blocks_fetched_distinct;
+  *out = o;
+}
+
 }  // namespace pts

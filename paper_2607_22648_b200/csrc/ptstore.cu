@@ -757,6 +757,14 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
   return PTSTORE_OK;
 }
 
+int ptstore_stats_enqueue(ptstore_t* h, ptstore_stats_t* out, ptstore_stream_t stream) {
+  static_assert(sizeof(StatsOut) == sizeof(ptstore_stats_t), "device and host views of the counters must match");
+  if (!h || !out) return PTSTORE_E_INVAL;
+  stats_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(h->st, h->epoch, reinterpret_cast<StatsOut*>(out));
+  PTS_CHECK_LAUNCH(h);
+  return PTSTORE_OK;
+}
+
 uint64_t ptstore_launch_count(const ptstore_t* h) { return h ? h->launches : 0; }
 int ptstore_last_cuda_error(const ptstore_t* h) { return h ? h->last_cuda : 0; }
 

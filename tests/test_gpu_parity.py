@@ -364,6 +364,12 @@ def test_edge_cases_and_errors():
     mo, io, _, _ = p.lookup([s], 4)
     assert mo.tolist() == [2]
     assert g.launch_count() > 10
+    # the non-blocking counters equal the blocking ones
+    buf = torch.zeros(__import__("ctypes").sizeof(G.Stats), dtype=torch.uint8).pin_memory()
+    g.stats_enqueue(buf)
+    torch.cuda.synchronize()
+    a, b = G.Stats.from_buffer_copy(buf.numpy().tobytes()), g.stats()
+    assert bytes(a) == bytes(b)
     p.close()
 
 
