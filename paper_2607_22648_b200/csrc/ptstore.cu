@@ -189,7 +189,7 @@ int launch_hash_split(ptstore* h, const int* tokens, const long long* offsets, i
 
 int lanes_for(const ptstore* h, int R, int max_blocks) {
   const u32 forced = (h->cfg.flags >> 8) & 0xFFu;
-  if (forced == 8 || forced == 16 || forced == 32) return (int)forced;
+  if (forced == 4 || forced == 8 || forced == 16 || forced == 32) return (int)forced;
   if (max_blocks <= 8 || R >= 4096) return 8;
   if (max_blocks <= 16 || R >= 1024) return 16;
   return 32;
@@ -547,6 +547,7 @@ int ptstore_hash(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, in
   u64* ko = reinterpret_cast<u64*>(keys_out);
   if (split_path(h, R, max_blocks)) return launch_hash_split(h, tokens, off, R, max_blocks, ko, s);
   switch (lanes_for(h, R, max_blocks)) {
+    case 4: return launch_hash<4>(h, tokens, off, R, max_blocks, ko, s);
     case 8: return launch_hash<8>(h, tokens, off, R, max_blocks, ko, s);
     case 16: return launch_hash<16>(h, tokens, off, R, max_blocks, ko, s);
     default: return launch_hash<32>(h, tokens, off, R, max_blocks, ko, s);
@@ -570,6 +571,7 @@ int ptstore_lookup(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
     return PTSTORE_OK;
   }
   switch (lanes_for(h, R, max_blocks)) {
+    case 4: return launch_lookup<4>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
     case 8: return launch_lookup<8>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
     case 16: return launch_lookup<16>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
     default: return launch_lookup<32>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
@@ -623,6 +625,7 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   const long long* off = reinterpret_cast<const long long*>(offsets);
   if (split_path(h, R, max_blocks)) rc = launch_hash_split(h, tokens, off, R, max_blocks, h->keys, s);
   else switch (lanes_for(h, R, max_blocks)) {
+    case 4: rc = launch_hash<4>(h, tokens, off, R, max_blocks, h->keys, s); break;
     case 8: rc = launch_hash<8>(h, tokens, off, R, max_blocks, h->keys, s); break;
     case 16: rc = launch_hash<16>(h, tokens, off, R, max_blocks, h->keys, s); break;
     default: rc = launch_hash<32>(h, tokens, off, R, max_blocks, h->keys, s); break;

@@ -49,3 +49,39 @@ def test_host_only_calls_validate_arguments():
     assert lib.ptstore_create(C.byref(cfg), C.byref(out), None) == -1 and not out.value
     assert lib.ptstore_strerror(-1) == b"invalid argument"
     assert lib.ptstore_strerror(0) == b"ok"
+
+
+def test_header_is_plain_c():
+    """The boundary is a C ABI: the header must compile as C99 with no other include than stdint.h."""
+    import subprocess
+    import tempfile
+    src = '#include "ptstore.h"\nint main(void) { ptstore_config_t c; c.struct_size = (uint32_t)sizeof c; return (int)(c.struct_size == 0) + PTSTORE_OK; }\n'
+    with tempfile.TemporaryDirectory() as d:
+        path = os.path.join(d, "t.c")
+        open(path, "w").write(src)
+        subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                               "-fsyntax-only", path])
+
+
+def test_ctypes_structs_match_the_c_layout():
+    """sizeof / offsetof of the structs the binding declares, checked against the C compiler."""
+    import subprocess
+    import tempfile
+    from paper_2607_22648_b200.binding import Config, PagedCache, Stats
+    prog = r'''
+#include <stdio.h>
+#include <stddef.h>
+#include "ptstore.h"
+int main(void) {
+  printf("%zu %zu %zu %zu %zu %zu\n", sizeof(ptstore_config_t), offsetof(ptstore_config_t, salt), offsetof(ptstore_config_t, table_slots),
+         offsetof(ptstore_config_t, device), sizeof(ptstore_paged_cache_t), sizeof(ptstore_stats_t));
+  return 0;
+}
+'''
+    with tempfile.TemporaryDirectory() as d:
+        path, exe = os.path.join(d, "t.c"), os.path.join(d, "t")
+        open(path, "w").write(prog)
+        subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), "-o", exe, path])
+        got = [int(x) for x in subprocess.check_output([exe]).split()]
+    want = [C.sizeof(Config), Config.salt.offset, Config.table_slots.offset, Config.device.offset, C.sizeof(PagedCache), C.sizeof(Stats)]
+    assert got == want

@@ -32,7 +32,7 @@ ENGINES = [
 ]
 
 
-@pytest.mark.parametrize("lanes", [0, 8, 16, 32])
+@pytest.mark.parametrize("lanes", [0, 4, 8, 16, 32])
 def test_hash_matches_oracle(lanes):
     Pair, dev, G = _imports()
     rng = np.random.default_rng(lanes)
@@ -244,7 +244,7 @@ def test_lookup_stress_small_matches_oracle():
     Pair, dev, G = _imports()
     ws = W.lookup_stress(n_roots=1500, n_queries=2048)
     sh = W.KVShape(1, 1, 8, 16)
-    for lanes in (8, 16, 32):
+    for lanes in (4, 8, 16, 32):
         p = Pair(sh, ws.n_nodes, flags=G.lookup_lanes(lanes), max_requests=2048, max_batch_blocks=2048 * 64,
                  table_slots=ws.table_slots, byte_mode=False)
         for i in range(0, len(ws.store_seqs), 2048):
