@@ -106,12 +106,12 @@ __global__ void __launch_bounds__(THREADS) copy_vector_kernel(Store st, Paged pc
         }
         e = (u32)nd.x;
       }
-      continue;
-    }
+    } else {
 #pragma unroll
-    for (int k = 0; k < UNROLL; ++k) {
-      const u64 o = ((u64)k * THREADS + threadIdx.x) * 16;
-      if (o < left) st_stream(dst + o, v[k]);
+      for (int k = 0; k < UNROLL; ++k) {
+        const u64 o = ((u64)k * THREADS + threadIdx.x) * 16;
+        if (o < left) st_stream(dst + o, v[k]);
+      }
     }
   }
 }
