@@ -66,8 +66,8 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 #define PTSTORE_PINNED_LIST 0x1u  /* the id list passed in was produced by a lookup with PTSTORE_PIN */
 
 /* flags of ptstore_config_t */
-#define PTSTORE_COPY_VECTOR  0x0u  /* copy engine: 16-byte vector loads/stores (always used for the host tier) */
-#define PTSTORE_COPY_BULK    0x1u  /* copy engine: bulk-async copies through a shared-memory ring (HBM<->HBM) */
+#define PTSTORE_COPY_BULK    0x0u  /* default copy engine for HBM<->HBM: bulk-async copies through a shared-memory ring */
+#define PTSTORE_COPY_VECTOR  0x1u  /* use 16-byte vector loads/stores everywhere (the host tier always uses them) */
 /* eviction order (Section 4.1 "Access pattern-aware eviction policy"): default is least recently used; with this
  * flag it is Greedy-Dual-Size-Frequency with one size and one cost per block: priority H = L + F, F = accesses of
  * the block (one per request that matched or stored it), L = the largest priority evicted so far.  Ties and the

@@ -14,7 +14,7 @@ OK, E_INVAL, E_CUDA, E_NOMEM, E_LIMIT = 0, -1, -2, -3, -4
 S_NOSPACE, S_TABLE_FULL, S_BOUNDS, S_STATE, S_TIMEOUT = 1, 2, 4, 8, 16
 PIN, NO_TOUCH = 1, 2
 PINNED_LIST = 1
-COPY_VECTOR, COPY_BULK = 0, 1
+COPY_BULK, COPY_VECTOR = 0, 1
 EVICT_GDSF = 2
 TIER_HBM, TIER_HOST = 0, 1
 

@@ -286,7 +286,7 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
   }
   const u32 variant = (h->cfg.flags >> 16) & 0xFu;
   int per_sm = (int)((h->cfg.flags >> 20) & 0xFFu);
-  if ((h->cfg.flags & PTSTORE_COPY_BULK) && !host_side_possible) {
+  if (!(h->cfg.flags & PTSTORE_COPY_VECTOR) && !host_side_possible) {
     BulkVariant v = kBulkVariants[variant < (u32)kNumBulkVariants ? variant : 0];
     if (v.stages == 0) v = auto_bulk(h->st.chunk_bytes);
     if (h->has_env_tune) v = h->env_tune;
