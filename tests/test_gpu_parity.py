@@ -461,3 +461,63 @@ def test_degenerate_shapes():
     p.lookup(many, 2)
     p.check_counts(); assert p.check_status() == 0
     p.close()
+
+
+def test_random_histories_across_all_option_combinations():
+    """Tiers x eviction policy x (a)synchronous demotion x copy engine, with promotion, held pins and random evictions:
+    every call compared with the oracle, pools compared every 20 steps."""
+    import itertools
+    Pair, dev, G = _imports()
+    sh = W.KVShape(2, 1, 8, 2)
+    B = 2
+    runs = 0
+    for seed, (host, policy, asyn, engine) in itertools.product(range(3), itertools.product((0, 30), ("lru", "gdsf"), (False, True),
+                                                                                          ("vector", "bulk"))):
+        if asyn and not host:
+            continue
+        rng = np.random.default_rng(2000 + seed)
+        p = Pair(sh, 48, host_blocks=host, salt=seed, flags=G.COPY_VECTOR if engine == "vector" else G.COPY_BULK, max_requests=8,
+                 max_batch_blocks=8 * 14, table_slots=509, policy=policy)
+        seqs, held = [], []
+        for step in range(60):
+            base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.8 else np.zeros(0, dtype=np.int32)
+            cut = int(rng.integers(0, len(base) + 1))
+            s = np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(1, 12)), dtype=np.int32)])[:28]
+            seqs.append(s)
+            batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(int(rng.integers(1, 7)))] + [s]
+            mb = 14
+            mo, io, _, _ = p.lookup(batch, mb, flags=1)
+            if host and rng.random() < 0.6:
+                io, _ = p.promote(io, mo, True, int(rng.integers(0, 8)))
+            nd = max(int(mo.sum()), 1) + 2
+            dst = [np.full((2, nd, sh.chunk_bytes), 7, dtype=np.uint8) for _ in range(sh.layers)]
+            bt = np.full((len(batch), mb), -1, dtype=np.int32)
+            perm, k = rng.permutation(nd), 0
+            for r in range(len(batch)):
+                for j in range(mo[r]):
+                    bt[r, j] = perm[k]
+                    k += 1
+            tier = int(rng.integers(0, 2)) if host else 0
+            n_ev = int(rng.integers(0, 16))
+            do_ev = rng.random() < 0.75
+            if asyn and do_ev:
+                p.evict(tier, n_ev, literal=False, asynchronous=True)
+            p.fetch(io, mo, dst, bt)
+            if not asyn and do_ev:
+                p.evict(tier, n_ev, literal=bool(step % 2))
+            need = sum(len(x) // B for x in batch)
+            src = W.random_kv_cache(seed * 1000 + step, sh, need + 1)
+            p.insert(batch, mb, src, W.shuffled_block_tables(rng, batch, B, mb, need + 1))
+            if rng.random() < 0.8:
+                p.release(io, mo)
+            else:
+                held.append((io, mo))
+            if held and rng.random() < 0.4:
+                p.release(*held.pop())
+            p.check_status()
+            if step % 20 == 19:
+                p.check_pools()
+                p.check_counts()
+        p.close()
+        runs += 1
+    assert runs == 36
