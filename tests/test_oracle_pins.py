@@ -616,3 +616,32 @@ def test_gdsf_literal_loop_equals_sorted_form_and_priorities_are_monotone(host):
                     assert nodes[nd["parent"]]["refcount"] >= nd["refcount"]
             logs.append(log)
         assert logs[0] == logs[1], seed
+
+
+def test_mix_avalanche():
+    """Flipping one input bit flips every output bit with probability close to one half."""
+    rng = np.random.default_rng(7)
+    trials = 4000
+    counts = np.zeros(64, dtype=np.int64)
+    for _ in range(trials):
+        x = int(rng.integers(0, 1 << 63)) | (int(rng.integers(0, 2)) << 63)
+        bit = int(rng.integers(0, 64))
+        d = H["mix"](x) ^ H["mix"](x ^ (1 << bit))
+        counts += np.array([(d >> b) & 1 for b in range(64)])
+    p = counts / trials
+    assert 0.45 < p.min() and p.max() < 0.55, (p.min(), p.max())
+
+
+def test_chained_keys_spread_evenly_over_a_table():
+    """Home slots floor(key * slots / 2^64) of 50,000 chained keys fill a 71,429-slot table like uniform draws would."""
+    rng = np.random.default_rng(8)
+    o = Oracle(1, 1, 8, 2, 16, 3, 4)
+    seqs = [rng.integers(0, 128000, size=16 * 10, dtype=np.int32) for _ in range(5000)]
+    keys = o.hash(*W.ragged(seqs), 10).ravel()
+    assert len(np.unique(keys)) == 50000
+    slots = 71429
+    home = np.array([(int(k) * slots) >> 64 for k in keys])
+    occupied = len(np.unique(home))
+    expect = slots * (1 - np.exp(-50000 / slots))                      # balls into bins
+    assert abs(occupied - expect) / expect < 0.01
+    assert np.bincount(home, minlength=slots).max() <= 8
