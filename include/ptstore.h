@@ -73,7 +73,7 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
  * the block (one per request that matched or stored it), L = the largest priority evicted so far.  Ties and the
  * leaves-first rule are as for LRU. */
 #define PTSTORE_EVICT_GDSF   0x2u
-/* tuning fields of flags (0 = library default): lanes per request of the lookup (8, 16 or 32),
+/* tuning fields of flags (0 = library default): lanes per request of the lookup (4, 8, 16 or 32),
  * copy-kernel variant, copy CTAs per SM */
 #define PTSTORE_LOOKUP_LANES(n)   (((uint32_t)(n) & 0xFFu) << 8)
 #define PTSTORE_COPY_VARIANT(v)   (((uint32_t)(v) & 0xFu) << 16)
@@ -85,7 +85,7 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 
 typedef struct {
   uint32_t struct_size;          /* sizeof(ptstore_config_t), checked */
-  uint32_t flags;                /* PTSTORE_COPY_* */
+  uint32_t flags;                /* PTSTORE_COPY_* | PTSTORE_EVICT_GDSF | tuning fields; 0 = defaults */
   uint32_t num_layers, num_kv_heads, head_dim, elem_bytes;   /* bf16: elem_bytes = 2 */
   uint32_t block_tokens;         /* tokens per block, >= 1 */
   uint32_t max_requests;         /* largest R any call will pass */
@@ -95,7 +95,8 @@ typedef struct {
   void*    host_pool;            /* device-visible pointer of mapped pinned memory, or NULL */
   uint32_t hbm_blocks;           /* >= 1 */
   uint32_t host_blocks;          /* 0 = no host tier */
-  uint64_t table_slots;          /* hash-table slots (any integer > hbm_blocks+host_blocks) */
+  uint64_t table_slots;          /* hash-table slots: any integer > hbm_blocks+host_blocks; for short probe runs use
+                                    about (hbm_blocks + host_blocks + largest insert batch) / 0.7 */
   void*    workspace;            /* device memory, 256-byte aligned */
   uint64_t workspace_bytes;      /* >= ptstore_workspace_bytes(cfg) */
   int32_t  device;               /* CUDA device ordinal that owns pools and workspace */
