@@ -521,3 +521,26 @@ def test_random_histories_across_all_option_combinations():
         p.close()
         runs += 1
     assert runs == 36
+
+
+def test_maximum_depth_request():
+    """max_blocks at its limit of 65,535: one request of 65,535 one-token blocks; the eviction order still puts the
+    deepest block first (the depth field of the sort key is 16 bits wide)."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    rng = np.random.default_rng(12)
+    seq = rng.integers(0, 50000, size=65535, dtype=np.int32)
+    p = Pair(sh, 70000, max_requests=2, max_batch_blocks=2 * 65535, byte_mode=False)
+    ids, newb = p.insert([seq], 65535)
+    assert newb.tolist() == [65535] and ids[0, -1] == 65534
+    mo, io, _, _ = p.lookup([seq, seq[:40000]], 65535, flags=1)
+    assert mo.tolist() == [65535, 40000]
+    p.release(io, mo)
+    ne, v = p.evict(0, 3)
+    assert v.tolist() == [65534, 65533, 65532]
+    with pytest.raises(G.PTStoreError) as e:
+        p.g.lookup(dev(seq), dev(np.array([0, 65535], dtype=np.int64)), 65536)
+    assert e.value.code == G.E_INVAL
+    p.check_counts()
+    assert p.check_status() == 0
+    p.close()
