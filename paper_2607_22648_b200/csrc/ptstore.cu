@@ -230,14 +230,17 @@ bool env_bulk_tune(BulkVariant* v) {
   return true;
 }
 
-// Default ring: stages of min(chunk, 32 KiB) and about 64 KiB of loads in flight per SM with one CTA per SM.
-// On B200 the copy was fastest with FEW bytes in flight (3 x 32 KiB x 1 CTA and 2 x 32 KiB x 2 CTAs per SM
-// both gave ~6.63 TB/s read+write on 32 KiB chunks; deeper rings and more CTAs were 3-7 % slower).
+// Default ring, from measurements on B200 (read+write GB/s of the fetch / insert copies on the bench workload):
+//   32 KiB chunks: 3 x 32 KiB x 1 CTA per SM 6.65 / 6.46 TB/s (deeper rings and more CTAs lose 3-7 %: few bytes in flight win)
+//   16 KiB chunks: 3 x 16 KiB x 2 CTAs       6.54 / 6.25       (1 CTA: 5.80 / 5.37 - one issuing thread per SM is too slow)
+//    8 KiB chunks: 3 x  8 KiB x 3 CTAs       6.47 / 6.21       (9 x 8 KiB x 1 CTA: 5.43 / 4.61)
+//    4 KiB chunks: 5 x  4 KiB x 4 CTAs       6.48 / 5.69
+// i.e. about 64 KiB of loads in flight per SM, spread over enough issuing threads that none has less than ~1 us per piece.
 BulkVariant auto_bulk(u64 chunk_bytes) {
-  int stage = (int)(chunk_bytes < 32768 ? chunk_bytes : 32768);
-  int stages = 1 + 65536 / stage;
-  if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
-  return {stages, stage, 1, 1, 0};
+  const int stage = (int)(chunk_bytes < 32768 ? chunk_bytes : 32768);
+  const int ctas = stage >= 32768 ? 1 : stage >= 16384 ? 2 : stage >= 8192 ? 3 : 4;
+  const int stages = stage >= 8192 ? 3 : 5;
+  return {stages, stage, ctas, 1, 0};
 }
 
 template <int MODE>
