@@ -17,14 +17,18 @@ namespace pts {
 template <int L>
 __device__ __forceinline__ u64 chain_chunk(u64& parent, u64 c, int lane, int steps) {
   const int sl = lane & (L - 1), base_lane = lane & ~(L - 1);
-  u64 k = parent, mine = 0;
+  u64 mine = 0;
   // the chain itself is serial (three dependent 64-bit multiplies per step); the shuffle that brings the next
-  // block's content hash is issued one step ahead so that its latency hides behind the arithmetic
+  // block's content hash is issued one step ahead so that its latency hides behind the arithmetic.  The remap of
+  // the reserved keys is kept off the dependent path: with x the un-remapped value, fix(x) * C1 = x * C1 + (x < 2 ?
+  // 2 * C1 : 0), so the multiply starts as soon as x exists and the compare runs beside it.
+  u64 x = parent;                                  // parent is a finished key (>= 2), so it is its own un-remapped value
   u64 ci = __shfl_sync(FULL, c, base_lane);
   for (int i = 0; i < steps; ++i) {
     const u64 cn = __shfl_sync(FULL, c, base_lane + ((i + 1) & (L - 1)));
-    k = hchain(k, ci);
-    if (sl == i) mine = k;
+    const u64 corr = x < 2 ? 2 * HC1 : 0;
+    x = hmix(x * HC1 + corr + ci);
+    if (sl == i) mine = hfix(x);
     ci = cn;
   }
   return mine;
