@@ -544,3 +544,32 @@ def test_maximum_depth_request():
     p.check_counts()
     assert p.check_status() == 0
     p.close()
+
+
+@pytest.mark.parametrize("engine", ["bulk", "vector"])
+def test_chunk_sizes_that_do_not_divide_into_stages(engine):
+    """Chunks of 48 KiB (a 32 KiB piece and a 16 KiB tail), 1600 B and 80 B: byte-exact insert and fetch."""
+    Pair, dev, G = _imports()
+    rng = np.random.default_rng(21)
+    for sh in (W.KVShape(2, 8, 128, 24), W.KVShape(3, 1, 8, 100), W.KVShape(2, 1, 8, 5)):
+        B = sh.block_tokens
+        p = Pair(sh, 40, flags=G.COPY_VECTOR if engine == "vector" else G.COPY_BULK, max_requests=8, max_batch_blocks=8 * 8)
+        base = rng.integers(0, 1000, size=6 * B + 3, dtype=np.int32)
+        seqs = [base, np.concatenate([base[:2 * B], rng.integers(0, 1000, size=3 * B, dtype=np.int32)]), base[:4 * B]]
+        need = sum(len(s) // B for s in seqs)
+        src = W.random_kv_cache(5, sh, need + 2)
+        p.insert(seqs, 8, src, W.shuffled_block_tables(rng, seqs, B, 8, need + 2))
+        p.check_pools()
+        mo, io, _, _ = p.lookup(seqs + [base], 8)
+        assert mo.tolist() == [6, 5, 4, 6]
+        nd = int(mo.sum()) + 3
+        dst = [np.full((2, nd, sh.chunk_bytes), 0x77, dtype=np.uint8) for _ in range(sh.layers)]
+        bt = np.full((4, 8), -1, dtype=np.int32)
+        perm, k = rng.permutation(nd), 0
+        for r in range(4):
+            for j in range(mo[r]):
+                bt[r, j] = perm[k]
+                k += 1
+        p.fetch(io, mo, dst, bt)
+        assert p.check_status() == 0
+        p.close()
