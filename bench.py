@@ -377,6 +377,9 @@ def run_gpu(args):
                    "batch": wl.batch, "eviction": args.policy, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
                    "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
+        # the same steps counted by the bytes DRAM has to move (a source block shared by several prompts is read once)
+        "value_on_needed_dram_bytes": round((main["distinct"] + main["fetched"] + 2 * (main["inserted"] + main["demoted"] + main["promoted"]))
+                                            * wl.sh.block_bytes / (main["ms"] * 1e-3) / 1e9, 1),
         "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_inserted": main["inserted"] / K, "blocks_dropped": main["dropped"] / K,
                      "hit_rate_blocks": round(main["matched"] / max(main["qblocks"], 1), 4),
                      "fetch_call_ms": round(fetch_ms / K, 4), "insert_call_ms": round(insert_ms / K, 4),
