@@ -79,16 +79,21 @@ __global__ void __launch_bounds__(256) collect_kernel(Store st, int tier, const 
 
 // ---- stable LSD radix sort of Key2, 8 bits per pass --------------------------------------------------------
 constexpr int SORT_THREADS = 256;
-constexpr int SORT_TILE = 2048;      // elements per CTA: 8 warps x 8 steps x 32 lanes
+// elements per CTA = 256 threads x STEPS: 512 (STEPS 2) for stores up to 32k blocks, so that a sort of a few ten thousand
+// candidates spreads over tens of SMs and each CTA's serial part stays short; 2048 (STEPS 8) beyond, to keep the
+// digit-by-tile histogram small
+constexpr int sort_steps_for(unsigned long long n_blocks) { return n_blocks <= (32u << 10) ? 2 : 8; }
 
 __device__ __forceinline__ u32 digit_of(const Key2& k, int word, int shift) { return (u32)(((word ? k.hi : k.lo) >> shift) & 0xFFu); }
 
+template <int STEPS>
 __global__ void __launch_bounds__(SORT_THREADS) sort_hist_kernel(const Key2* __restrict__ in, const u32* __restrict__ n_ptr, int word,
                                                                  int shift, u32* __restrict__ hist, u32 n_tiles) {
   __shared__ u32 h[256];
   h[threadIdx.x] = 0;
   __syncthreads();
   const u32 n = *n_ptr;
+  constexpr u32 SORT_TILE = SORT_THREADS * STEPS;
   const u32 base = blockIdx.x * SORT_TILE;
   for (u32 i = threadIdx.x; i < SORT_TILE; i += SORT_THREADS)
     if (base + i < n) atomicAdd(&h[digit_of(in[base + i], word, shift)], 1u);
@@ -123,10 +128,12 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(u32* __restrict__ hist,
   }
 }
 
+template <int STEPS>
 __global__ void __launch_bounds__(SORT_THREADS) sort_scatter_kernel(const Key2* __restrict__ in, Key2* __restrict__ out,
                                                                     const u32* __restrict__ n_ptr, int word, int shift,
                                                                     const u32* __restrict__ hist, u32 n_tiles) {
   __shared__ u32 wh[SORT_THREADS / 32][256];     // per-warp digit counts, then per-warp output cursors
+  constexpr u32 SORT_TILE = SORT_THREADS * STEPS;
   const u32 n = *n_ptr;
   const u32 tile0 = blockIdx.x * SORT_TILE;
   if (tile0 >= n) return;
@@ -134,7 +141,6 @@ __global__ void __launch_bounds__(SORT_THREADS) sort_scatter_kernel(const Key2* 
   for (int i = lane; i < 256; i += 32) wh[w][i] = 0;
   __syncwarp();
   const u32 seg = tile0 + w * (SORT_TILE / (SORT_THREADS / 32));
-  constexpr int STEPS = SORT_TILE / SORT_THREADS;
   Key2 el[STEPS];
   u32 dg[STEPS];
 #pragma unroll

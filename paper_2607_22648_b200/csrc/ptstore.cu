@@ -52,7 +52,8 @@ Layout make_layout(const ptstore_config_t* c) {
   L.ctrl = take(sizeof(Ctrl));
   L.blocked = take(N);
   L.sort[0] = take(N * sizeof(Key2)); L.sort[1] = take(N * sizeof(Key2));
-  L.n_tiles = (u32)((N + SORT_TILE - 1) / SORT_TILE);
+  const u64 sort_tile = (u64)SORT_THREADS * sort_steps_for(N);
+  L.n_tiles = (u32)((N + sort_tile - 1) / sort_tile);
   L.hist = take((u64)256 * L.n_tiles * 4);
   L.room = take((u64)c->host_blocks * 4);
   L.desc = take((M > N ? M : N) * sizeof(int2));
@@ -321,6 +322,7 @@ int bytes_needed(u64 max_value) {
 // sorts sort_buf[0][0..ev_cand) ; returns the index of the buffer that holds the result in *result
 int launch_sort(ptstore* h, cudaStream_t s, int* result) {
   const u32 nt = h->lay.n_tiles;
+  const bool small = sort_steps_for((u64)h->cfg.hbm_blocks + h->cfg.host_blocks) == 2;
   int cur = 0;
   struct Pass { int word, shift; } passes[16];
   int np = 0;
@@ -332,11 +334,14 @@ int launch_sort(ptstore* h, cudaStream_t s, int* result) {
   const int st_bytes = bytes_needed(h->st.policy ? h->epoch * (u64)h->cfg.max_requests : h->epoch);
   for (int b = 0; b < st_bytes; ++b) passes[np++] = {1, 8 * b};
   for (int p = 0; p < np; ++p) {
-    sort_hist_kernel<<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
+    if (small) sort_hist_kernel<2><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
+    else sort_hist_kernel<8><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
     PTS_CHECK_LAUNCH(h);
     sort_scan_kernel<<<1, 1024, 0, s>>>(h->hist, 256u * nt);
     PTS_CHECK_LAUNCH(h);
-    sort_scatter_kernel<<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], h->sort_buf[cur ^ 1], &h->st.ctrl->ev_cand, passes[p].word,
+    if (small) sort_scatter_kernel<2><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], h->sort_buf[cur ^ 1], &h->st.ctrl->ev_cand, passes[p].word,
+                                                                passes[p].shift, h->hist, nt);
+    else sort_scatter_kernel<8><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], h->sort_buf[cur ^ 1], &h->st.ctrl->ev_cand, passes[p].word,
                                                      passes[p].shift, h->hist, nt);
     PTS_CHECK_LAUNCH(h);
     cur ^= 1;
