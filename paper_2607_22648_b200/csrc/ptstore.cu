@@ -330,8 +330,9 @@ int launch_sort(ptstore* h, cudaStream_t s, int* result) {
   for (int b = 0; b < id_bytes; ++b) passes[np++] = {0, 8 * b};
   passes[np++] = {0, 32};
   passes[np++] = {0, 40};
-  // LRU: stamps are at most the epoch.  GDSF: a priority is at most the number of accesses ever counted
-  const int st_bytes = bytes_needed(h->st.policy ? h->epoch * (u64)h->cfg.max_requests : h->epoch);
+  // LRU: stamps are at most the epoch.  GDSF: a priority H = L + F has no bound the host knows (L accumulates the
+  // priorities of earlier victims), so the whole word is sorted
+  const int st_bytes = h->st.policy ? 8 : bytes_needed(h->epoch);
   for (int b = 0; b < st_bytes; ++b) passes[np++] = {1, 8 * b};
   for (int p = 0; p < np; ++p) {
     if (small) sort_hist_kernel<2><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);

@@ -22,7 +22,7 @@ ENGINES = [
     ("vector", lambda G: G.COPY_VECTOR),
     ("vector_u8", lambda G: G.COPY_VECTOR | G.copy_variant(1)),
     ("vector_512", lambda G: G.COPY_VECTOR | G.copy_variant(2)),
-    ("bulk_6x16k", lambda G: G.COPY_BULK),
+    ("bulk_auto", lambda G: G.COPY_BULK),
     ("bulk_8x8k_3cta", lambda G: G.COPY_BULK | G.copy_variant(1)),
     ("bulk_3x32k", lambda G: G.COPY_BULK | G.copy_variant(2)),
     ("bulk_12x16k", lambda G: G.COPY_BULK | G.copy_variant(5)),
@@ -238,6 +238,54 @@ def test_gdsf_keeps_frequent_blocks_that_lru_would_evict():
         p.check_counts()
         p.close()
     assert out["lru"] == [1, 0] and out["gdsf"] == [3, 2]
+
+
+def test_gdsf_priority_above_calls_times_requests_is_ordered_whole():
+    """A block's priority H = L + F reaches 256 after 3 calls of 64 requests: the eviction order has to take the whole
+    priority into account, or the hot parent is taken before the cold leaf."""
+    Pair, dev, G = _imports()
+    p = Pair(W.KVShape(1, 1, 8, 2), 8, max_requests=64, max_batch_blocks=128, policy="gdsf")
+    bv = np.array([1, 1, 2, 2], dtype=np.int32)
+    b = bv[:2]
+    p.insert([bv] * 64, 2)
+    mo, io, _, _ = p.lookup([b] * 64, 2, flags=1)
+    ne, v = p.evict(0, 1)
+    assert v.tolist() == [1]
+    p.lookup([b] * 64, 2)
+    p.release(io, mo)
+    p.insert([np.array([1, 1, 3, 3], dtype=np.int32)], 2)
+    s = p.check_counts()
+    assert s.gdsf_clock == 64 and p.o.block_info(0)["last_use"] == 257
+    ne, v = p.evict(0, 1)
+    assert v.tolist() == [2]
+    ne, v = p.evict(0, 1)
+    assert v.tolist() == [0]
+    assert p.check_counts().gdsf_clock == 257
+    assert p.check_status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("host", [0, 4])
+def test_gdsf_long_history_of_single_requests_lockstep(host):
+    """One request per call (max_requests 1) for 300 steps: priorities outgrow the call count; victims compared in order."""
+    from tests.histories import small_request_gdsf_history
+    Pair, dev, G = _imports()
+    p = Pair(W.KVShape(1, 1, 8, 1), 6, host_blocks=host, max_requests=1, max_batch_blocks=4, policy="gdsf", table_slots=23)
+    worst = 0
+    for k, (op, arg) in enumerate(small_request_gdsf_history(300)):
+        if op == "lookup":
+            p.lookup([arg], 4)
+        elif op == "insert":
+            p.insert([arg], 4)
+        else:
+            p.evict(0, arg, literal=bool(k % 2))
+        worst = max([worst] + [p.o.block_info(i)["last_use"] - p.o.epoch() for i in range(6 + host) if p.o.block_info(i)["live"]])
+        if k % 50 == 49:
+            p.check_counts()
+    assert worst > 0
+    p.check_counts()
+    p.check_status()
+    p.close()
 
 
 def test_lookup_stress_small_matches_oracle():

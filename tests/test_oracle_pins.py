@@ -16,6 +16,7 @@ import pytest
 
 from oracle import Oracle, hash_parts, PIN, NO_TOUCH, S_NOSPACE, S_STATE
 from paper_2607_22648_b200 import workloads as W
+from tests.histories import small_request_gdsf_history
 
 M64 = (1 << 64) - 1
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hash_kat.txt")
@@ -577,6 +578,47 @@ def test_gdsf_keeps_frequent_blocks_that_lru_would_evict():
             assert o.block_info(4)["last_use"] == 2 and o.block_info(4)["freq"] == 1
     assert out["lru"] == [1, 0]                             # least recently used: the hot pair goes
     assert out["gdsf"] == [3, 2]                            # least frequently used: the cold pair goes, deeper first
+
+
+def test_gdsf_priority_grows_past_the_accesses_of_any_one_block():
+    """H = L + F with L itself a sum of earlier victims' priorities: a hand-worked history in which a block's priority
+    (256) exceeds calls x requests per call (3 x 64 = 192), so no bound built from the access count alone holds it."""
+    o = Oracle(1, 1, 8, 2, 2, 0, 8, policy="gdsf")
+    bv = np.array([1, 1, 2, 2], dtype=np.int32)             # blocks B (id 0) and V (id 1)
+    b = bv[:2]
+    o.insert(*W.ragged([bv] * 64), 2)                       # call 1: 64 requests store B and V: F = 64, H = 0 + 64 each
+    assert [o.block_info(i)["last_use"] for i in (0, 1)] == [64, 64]
+    m, ids = o.lookup(*W.ragged([b] * 64), 2, PIN)          # call 2: B asked for 64 times and pinned: F = 128, H = 128
+    assert o.block_info(0)["last_use"] == 128 and o.block_info(0)["refcount"] == 64
+    ne, v = o.evict(0, 1)                                   # only V is evictable: L = H(V) = 64
+    assert v.tolist() == [1] and o.inflation() == 64
+    o.lookup(*W.ragged([b] * 64), 2)                        # call 3: F = 192, H = L + F = 64 + 192
+    assert o.epoch() == 3 and o.block_info(0)["freq"] == 192 and o.block_info(0)["last_use"] == 256
+    o.release(ids, m)
+    bw = np.array([1, 1, 3, 3], dtype=np.int32)
+    o.insert(*W.ragged([bw]), 2)                            # W (id 2): F = 1, H = 65; B: F = 193, H = 257
+    assert o.block_info(2)["last_use"] == 65 and o.block_info(0)["last_use"] == 257
+    ne, v = o.evict(0, 1)
+    assert v.tolist() == [2] and o.inflation() == 65        # the leaf with the low priority goes, not the hot parent
+    ne, v = o.evict(0, 1)
+    assert v.tolist() == [0] and o.inflation() == 257
+
+
+def test_gdsf_priority_exceeds_the_call_count_in_a_long_single_request_history():
+    o = Oracle(1, 1, 8, 2, 1, 0, 6, policy="gdsf")
+    worst = 0
+    for op, arg in small_request_gdsf_history(300):
+        if op == "lookup":
+            o.lookup(*W.ragged([arg]), 4)
+        elif op == "insert":
+            o.insert(*W.ragged([arg]), 4)
+        else:
+            o.evict(0, arg)
+        for i in range(6):
+            nd = o.block_info(i)
+            if nd["live"]:
+                worst = max(worst, nd["last_use"] - o.epoch())
+    assert worst > 0                                        # some live priority was above calls x 1 request per call
 
 
 @pytest.mark.parametrize("host", [0, 40])
