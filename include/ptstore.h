@@ -16,6 +16,8 @@
  *     valid once the stream has reached that point.  Calls on one handle must be issued from one
  *     host thread at a time and onto one stream (or streams the caller has ordered); the library
  *     takes no lock.
+ *   - ptstore_create makes cfg->device the calling thread's current CUDA device and leaves it so; every later call on
+ *     the handle must be made with that device current (the library does not switch devices per call).
  *   - Return value: PTSTORE_OK (0) or a negative PTSTORE_E_* code for conditions the host can see
  *     (bad arguments, CUDA launch errors).  Conditions only the device can see (pool exhausted,
  *     table full, block-table entry out of range, refcount underflow) are OR-ed as PTSTORE_S_* bits
@@ -56,7 +58,12 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 #define PTSTORE_S_TABLE_FULL  0x2u   /* insert/rebuild: no free slot found within table_slots probes */
 #define PTSTORE_S_BOUNDS      0x4u   /* a block id or block-table entry was out of range; access skipped */
 #define PTSTORE_S_STATE       0x8u   /* release would have driven a refcount below zero; skipped */
-#define PTSTORE_S_TIMEOUT     0x10u  /* a bounded wait inside a copy kernel expired; that CTA stopped copying */
+#define PTSTORE_S_TIMEOUT     0x10u  /* a bounded wait inside a kernel expired (a copy CTA stopped copying, or a grid-wide
+                                        barrier gave up); the call's results are incomplete, the handle stays usable for
+                                        copies, and nothing is left running */
+#define PTSTORE_S_INFLIGHT    0x20u  /* fetch: a host-tier block named by the call was demoted by ptstore_evict_async /
+                                        ptstore_reserve(PTSTORE_ASYNC_COPY) and its copy has not been joined yet; that
+                                        entry was skipped */
 
 /* flags of ptstore_lookup */
 #define PTSTORE_PIN       0x1u   /* refcount++ on every matched (request, block) pair */
@@ -73,11 +80,23 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
  * the block (one per request that matched or stored it), L = the largest priority evicted so far.  Ties and the
  * leaves-first rule are as for LRU. */
 #define PTSTORE_EVICT_GDSF   0x2u
-/* tuning fields of flags (0 = library default): lanes per request of the lookup (4, 8, 16 or 32),
- * copy-kernel variant, copy CTAs per SM */
+/* tuning fields of flags (0 = library default):
+ *   PTSTORE_LOOKUP_LANES(n)      lanes per request of lookup / hash: 4, 8, 16 or 32
+ *   PTSTORE_COPY_CTAS_PER_SM(c)  CTAs per SM of the HBM<->HBM copy kernels
+ *   PTSTORE_COPY_VARIANT(v)      geometry of the copy kernels.  With PTSTORE_COPY_BULK, the ring of shared-memory stages:
+ *                                  0 sized from the chunk size (3 stages of min(chunk, 32 KiB), 1-4 CTAs per SM)
+ *                                  1 8 x 8 KiB, 3 CTAs per SM      2 3 x 32 KiB          3 4 x 16 KiB, 3 CTAs per SM
+ *                                  4 12 x 16 KiB                   5 6 x 16 KiB, two consecutive pieces per turn
+ *                                  6 6 x 16 KiB with evict-first L2 hints on loads and stores     7 3 x 64 KiB
+ *                                With PTSTORE_COPY_VECTOR, threads x 16-byte loads in flight per thread:
+ *                                  0 256 x 4, 16 CTAs per SM       1 256 x 8, 8 CTAs per SM       2 512 x 4, 4 CTAs per SM
+ *                                Other values select 0. */
 #define PTSTORE_LOOKUP_LANES(n)   (((uint32_t)(n) & 0xFFu) << 8)
 #define PTSTORE_COPY_VARIANT(v)   (((uint32_t)(v) & 0xFu) << 16)
 #define PTSTORE_COPY_CTAS_PER_SM(c) (((uint32_t)(c) & 0xFFu) << 20)
+
+/* flags of ptstore_reserve */
+#define PTSTORE_ASYNC_COPY  0x1u  /* run the demotion copy on the library's side stream, as ptstore_evict_async does */
 
 /* tiers of ptstore_evict */
 #define PTSTORE_TIER_HBM   0
@@ -95,8 +114,9 @@ typedef struct {
   void*    host_pool;            /* device-visible pointer of mapped pinned memory, or NULL */
   uint32_t hbm_blocks;           /* >= 1 */
   uint32_t host_blocks;          /* 0 = no host tier */
-  uint64_t table_slots;          /* hash-table slots: any integer > hbm_blocks+host_blocks; for short probe runs use
-                                    about (hbm_blocks + host_blocks + largest insert batch) / 0.7 */
+  uint64_t table_slots;          /* hash-table slots: any integer > hbm_blocks+host_blocks (values below 8 are raised to
+                                    8); for short probe runs use about (hbm_blocks + host_blocks + largest insert
+                                    batch) / 0.7 */
   void*    workspace;            /* device memory, 256-byte aligned */
   uint64_t workspace_bytes;      /* >= ptstore_workspace_bytes(cfg) */
   int32_t  device;               /* CUDA device ordinal that owns pools and workspace */
@@ -177,6 +197,19 @@ int ptstore_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets,
                    ptstore_stream_t stream);
 
 /*
+ * ptstore_lookup followed by ptstore_fetch of what it matched, as one call (Section 4.1: a load first finds the longest
+ * common prefix and then brings each of its tensors to the GPU pointers the application supplies; what matters to the
+ * application is the latency of the pair).  Same results as the two calls: matched_blocks and block_ids are written
+ * as by ptstore_lookup(flags), and every matched block j of request r is copied to cache block
+ * block_tables[r*max_blocks+j] as by ptstore_fetch.  The lookup kernel builds the copy lists itself while it probes,
+ * so the pair costs two kernel launches (three when requests are few and long, three or four with a host tier).
+ */
+int ptstore_lookup_fetch(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                         uint32_t flags, const ptstore_paged_cache_t* dst /*host struct*/,
+                         const int32_t* block_tables /*[R*max_blocks]*/, int32_t* matched_blocks /*[R]*/,
+                         int32_t* block_ids /*[R*max_blocks]*/, ptstore_stream_t stream);
+
+/*
  * Load (Section 4.1: iterate over the ids of an object and bring each tensor to the GPU pointers
  * the application supplies).  For every r, j < matched_blocks[r], layer l, s in {K,V}: copy one chunk
  * from pool block block_ids[r*max_blocks+j] to block block_tables[r*max_blocks+j] of the paged cache.
@@ -239,10 +272,25 @@ int ptstore_evict(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evic
  * ptstore_join on this handle.  It is NOT ordered with later ptstore_fetch calls: until the next of the calls just
  * named, fetch only block ids that were pinned (ptstore_lookup with PTSTORE_PIN) before this call — a pinned block
  * is never a victim, so such a fetch cannot touch a block in flight.  Without a host tier, or for tier HOST, this
- * is ptstore_evict.  The first call creates the stream and two events (no device memory).
+ * is ptstore_evict.  The first call creates the stream and two events (no device memory).  A fetch that names a
+ * host-tier block whose copy is still in flight skips that entry and raises PTSTORE_S_INFLIGHT.
  */
 int ptstore_evict_async(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids,
                         ptstore_stream_t stream);
+
+/*
+ * Make room before a store, decided on the device (Section 1: blocks of finished requests are evicted when space is
+ * needed; this is ptstore_evict(PTSTORE_TIER_HBM, n) with n computed where the free count lives, so the host need not
+ * wait for a lookup's result before it can queue the eviction):
+ *     n = max(0, want_free - sum(max(minus[i], 0), i < n_minus) - free HBM blocks),  capped at max_victims.
+ * Typical use: want_free = full blocks of the batch, minus = the matched_blocks array the preceding lookup wrote.
+ *   flags       0, or PTSTORE_ASYNC_COPY (the demotion copy runs as in ptstore_evict_async; same ordering rules)
+ *   n_evicted   out, device [2], as for ptstore_evict
+ *   victim_ids  out, device [2*max_victims] or NULL (then max_victims is ignored), as for ptstore_evict
+ * n_minus may not exceed max_requests (PTSTORE_E_LIMIT).
+ */
+int ptstore_reserve(ptstore_t* st, int64_t want_free, const int32_t* minus, int32_t n_minus, uint32_t flags,
+                    int32_t* n_evicted, int32_t* victim_ids, int32_t max_victims, ptstore_stream_t stream);
 
 /* Make `stream` wait for a demotion copy left running by ptstore_evict_async (no-op if there is none). */
 int ptstore_join(ptstore_t* st, ptstore_stream_t stream);
@@ -264,7 +312,11 @@ int ptstore_join(ptstore_t* st, ptstore_stream_t stream);
 int ptstore_promote(ptstore_t* st, int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
                     uint32_t flags, int32_t max_promote, int32_t* n_promoted, ptstore_stream_t stream);
 
-/* Synchronise `stream`, read the device status word into *status_out (host) and clear it. */
+/*
+ * Synchronise `stream`, read the device status word into *status_out (host) and clear it.  The read and the clear
+ * are two operations enqueued on `stream`: a bit raised by work running on ANOTHER stream between them is lost, so
+ * keep everything on one stream (or ordered) around this call.
+ */
 int ptstore_status(ptstore_t* st, ptstore_stream_t stream, uint32_t* status_out /*host*/);
 
 /* Synchronise `stream` and copy the counters to *out (host). */
@@ -277,6 +329,24 @@ int ptstore_stats(ptstore_t* st, ptstore_stream_t stream, ptstore_stats_t* out /
  * lookup while the fetch that follows is already running.
  */
 int ptstore_stats_enqueue(ptstore_t* st, ptstore_stats_t* out /*device-accessible*/, ptstore_stream_t stream);
+
+/*
+ * Polls a copy kernel spends on one wait for a load, in its main loop, before its CTA gives up, raises
+ * PTSTORE_S_TIMEOUT, waits (with the full built-in limit) for the loads it still has in flight and returns; 0 restores
+ * the built-in limit.  No paper counterpart.  Meant for failure-detection tests: a limit of 1 is a single test that
+ * never suspends, so a CTA whose first load has not landed yet gives up at once, without anything hanging or
+ * faulting, and the give-up-and-drain path can be exercised on a healthy GPU.
+ */
+int ptstore_set_wait_limit(ptstore_t* st, uint32_t polls);
+
+/*
+ * Measurement aid (no paper counterpart): the next copy kernel the handle launches for HBM-resident data (the gather of
+ * ptstore_fetch / ptstore_lookup_fetch, the scatter of ptstore_insert; not the small-grid host-link copies) gets
+ * `before` recorded on its stream just ahead of it and `after` just behind it.  Both are cudaEvent_t created by the
+ * caller with timing enabled; one shot.  cudaEventElapsedTime(before, after) is then the duration of that kernel alone,
+ * which is what a bandwidth figure for the copy engine has to be divided by.
+ */
+int ptstore_time_next_copy(ptstore_t* st, void* before /*cudaEvent_t*/, void* after /*cudaEvent_t*/);
 
 /* Number of this library's kernels launched through the handle so far (host counter, no sync). */
 uint64_t ptstore_launch_count(const ptstore_t* st);
@@ -297,7 +367,8 @@ int ptstore_last_cuda_error(const ptstore_t* st);
  * on every GPU that loads it, held until process exit.  Limits: R <= PTSTORE_STATIC_MAX_REQUESTS and
  * R*max_blocks <= PTSTORE_STATIC_MAX_PAIRS, else PTSTORE_E_LIMIT.  All calls on a GPU share that array: calls
  * that overlap on the GPU race, so keep them on one stream or order them.  The first call on each device
- * (made with that device current) looks up the array's address; issue it before any stream capture.
+ * (made with that device current) looks up the array's address; issue it before any stream capture, and do not make
+ * the first calls for one device from two host threads at once (the lookup is cached without a lock).
  * Calls no cudaMalloc / cudaFree / allocating routine.  Enqueues on `stream` and returns.
  */
 #define PTSTORE_STATIC_MAX_REQUESTS   1024u

@@ -11,9 +11,10 @@ import torch
 from . import build as _build
 
 OK, E_INVAL, E_CUDA, E_NOMEM, E_LIMIT = 0, -1, -2, -3, -4
-S_NOSPACE, S_TABLE_FULL, S_BOUNDS, S_STATE, S_TIMEOUT = 1, 2, 4, 8, 16
+S_NOSPACE, S_TABLE_FULL, S_BOUNDS, S_STATE, S_TIMEOUT, S_INFLIGHT = 1, 2, 4, 8, 16, 32
 PIN, NO_TOUCH = 1, 2
 PINNED_LIST = 1
+ASYNC_COPY = 1
 COPY_BULK, COPY_VECTOR = 0, 1
 EVICT_GDSF = 2
 TIER_HBM, TIER_HOST = 0, 1
@@ -57,7 +58,8 @@ class Stats(C.Structure):
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
-           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join", "ptstore_stats_enqueue"]
+           "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join", "ptstore_stats_enqueue", "ptstore_lookup_fetch",
+           "ptstore_reserve", "ptstore_set_wait_limit", "ptstore_time_next_copy"]
 
 
 def _load():
@@ -73,6 +75,10 @@ def _load():
     lib.ptstore_hash.argtypes = [vp, vp, vp, i32, i32, vp, vp]
     lib.ptstore_lookup.argtypes = [vp, vp, vp, i32, i32, u32, vp, vp, vp]
     lib.ptstore_fetch.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp]
+    lib.ptstore_lookup_fetch.argtypes = [vp, vp, vp, i32, i32, u32, C.POINTER(PagedCache), vp, vp, vp, vp]
+    lib.ptstore_reserve.argtypes = [vp, C.c_int64, vp, i32, u32, vp, vp, i32, vp]
+    lib.ptstore_set_wait_limit.argtypes = [vp, u32]
+    lib.ptstore_time_next_copy.argtypes = [vp, vp, vp]
     lib.ptstore_insert.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
     lib.ptstore_release.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.ptstore_evict.argtypes = [vp, i32, i32, vp, vp, vp]
@@ -213,6 +219,33 @@ class PTStore:
         R, mb = ids.shape
         self._check(lib.ptstore_fetch(self.h, _ptr(ids), _ptr(matched), R, mb, C.byref(cache.desc), _ptr(block_tables),
                                       _stream()), "ptstore_fetch")
+
+    def lookup_fetch(self, tokens, offsets, max_blocks, cache, block_tables, flags=0, matched=None, ids=None):
+        R = offsets.numel() - 1
+        if matched is None:
+            matched = torch.empty(R, dtype=torch.int32, device=self.device)
+        if ids is None:
+            ids = torch.empty((R, max_blocks), dtype=torch.int32, device=self.device)
+        self._check(lib.ptstore_lookup_fetch(self.h, _ptr(tokens), _ptr(offsets), R, max_blocks, flags, C.byref(cache.desc),
+                                             _ptr(block_tables), _ptr(matched), _ptr(ids), _stream()), "ptstore_lookup_fetch")
+        return matched, ids
+
+    def reserve(self, want_free, minus=None, flags=0, max_victims=0, n_evicted=None, victims=None):
+        """Evicts max(0, want_free - sum(minus) - free HBM blocks) blocks from HBM, decided on the device."""
+        if n_evicted is None:
+            n_evicted = torch.zeros(2, dtype=torch.int32, device=self.device)
+        if victims is None and max_victims:
+            victims = torch.full((2 * max_victims,), -1, dtype=torch.int32, device=self.device)
+        self._check(lib.ptstore_reserve(self.h, int(want_free), _ptr(minus), minus.numel() if minus is not None else 0, flags,
+                                        _ptr(n_evicted), _ptr(victims), max_victims, _stream()), "ptstore_reserve")
+        return n_evicted, victims
+
+    def time_next_copy(self, before, after):
+        """before / after: torch.cuda.Event(enable_timing=True) that have been recorded once (so that they exist)."""
+        self._check(lib.ptstore_time_next_copy(self.h, before.cuda_event, after.cuda_event), "ptstore_time_next_copy")
+
+    def set_wait_limit(self, polls):
+        self._check(lib.ptstore_set_wait_limit(self.h, polls), "ptstore_set_wait_limit")
 
     def insert(self, tokens, offsets, max_blocks, cache=None, block_tables=None, ids=None, new_blocks=None):
         R = offsets.numel() - 1

@@ -23,9 +23,10 @@ constexpr u64 KEY_EMPTY = 0ull;
 constexpr u64 KEY_TOMB = 1ull;
 constexpr u32 NO_ID = 0xFFFFFFFFu;
 constexpr u32 NO_SLOT = 0xFFFFFFFFu;
+constexpr u32 LINK_NIL = 0xFFFFFFFFu;  // end of a destination list (fetch)
 
 // ---- status bits / flags (mirror include/ptstore.h) -------------------------------------------------
-constexpr u32 S_NOSPACE = 1u, S_TABLE_FULL = 2u, S_BOUNDS = 4u, S_STATE = 8u, S_TIMEOUT = 16u;
+constexpr u32 S_NOSPACE = 1u, S_TABLE_FULL = 2u, S_BOUNDS = 4u, S_STATE = 8u, S_TIMEOUT = 16u, S_INFLIGHT = 32u;
 constexpr u32 F_PIN = 1u, F_NO_TOUCH = 2u;
 
 // ---- control block in device memory ----------------------------------------------------------------
@@ -51,7 +52,16 @@ struct Ctrl {
   u32 ev_host_dropped;  // evict: host-tier drops that made room for a demotion
   u32 live[2];
   u32 tombstones;
-  u32 work_counter;     // fetch: next work unit to hand out (dynamic dealing inside the copy kernel)
+  u32 work_counter;     // spare
+  // fetch: per-call scalars, double buffered by the call's sequence number so that no launch is needed to clear them:
+  // call k uses entry k & 1 and zeroes entry (k + 1) & 1 for the call after it
+  u32 f_pairs[2];       // distinct HBM-tier source blocks = entries of the descriptor list
+  u32 f_pairs_host[2];  // distinct host-tier source blocks (a descriptor list of their own)
+  u32 f_work[2];        // next work unit to hand out (dynamic dealing inside the copy kernel)
+  u32 pad1[2];
+  // arrival counters of the grid-wide barriers of cooperative kernels: launch k uses entry k % BAR_SLOTS and zeroes
+  // the entry half a ring ahead, so a counter is always zero when its turn comes, whatever happened to earlier launches
+  u32 bar[64];
   // cumulative counters
   u64 query_blocks, probes_issued, slots_visited, blocks_matched;   // totals are these plus the stripes below
   u64 blocks_fetched[2];
@@ -78,6 +88,7 @@ struct Store {
   u32* m_freq;          // GDSF policy: access count F
   u32* m_ref;
   u32* m_depth;
+  u32* m_flight;        // host-tier blocks: tag of the asynchronous demotion that last wrote the block (0 = none)
   int* ring_ids[2];
   u32 n[2];             // blocks per tier
   Ctrl* ctrl;
@@ -221,6 +232,45 @@ __device__ __forceinline__ unsigned char* block_ptr(const Store& st, u32 id) {
 }
 
 __device__ __forceinline__ void raise(const Store& st, u32 bit) { atomicOr(&st.ctrl->status, bit); }
+
+// ---- grid-wide barrier for cooperative launches ---------------------------------------------------------------------
+// All CTAs of a cooperative launch are resident at once, so they may wait for one another.  Every CTA calls sync() the
+// same number of times; the k-th call returns once all CTAs have made their k-th call.  The wait is bounded: after
+// GRID_POLL_LIMIT polls the CTA raises S_TIMEOUT and sync() returns false from then on without waiting (callers stop
+// touching shared state and fall through to the end of the kernel).
+constexpr int BAR_SLOTS = 64;
+constexpr u32 GRID_POLL_LIMIT = 1u << 24;
+struct GridBarrier {
+  u32* counter;
+  u32 arrived;      // arrivals expected by the end of the next sync(): gridDim.x * (calls so far + 1)
+  bool ok;
+  __device__ __forceinline__ void init(Ctrl* c, u32 launch_seq) {
+    counter = &c->bar[launch_seq % BAR_SLOTS];
+    arrived = 0;
+    ok = true;
+    if (blockIdx.x == 0 && threadIdx.x == 0) c->bar[(launch_seq + BAR_SLOTS / 2) % BAR_SLOTS] = 0;
+  }
+  __device__ __forceinline__ bool sync(const Store& st) {
+    arrived += gridDim.x;
+    if (gridDim.x == 1) { __syncthreads(); return ok; }
+    __syncthreads();
+    if (threadIdx.x == 0 && ok) {
+      __threadfence();
+      atomicAdd(counter, 1u);
+      u32 polls = 0;
+      while (true) {
+        u32 seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+        if (seen >= arrived) break;
+        if (++polls >= GRID_POLL_LIMIT) { ok = false; raise(st, S_TIMEOUT); break; }
+        __nanosleep(32);
+      }
+      __threadfence();
+    }
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    return ok;
+  }
+};
 
 // `count` accesses to block `id` in the call with stamp `epoch` (paper Section 1: LRU; Section 4.1 "Access
 // pattern-aware eviction policy": frequency-aware Greedy-Dual-Size-Frequency, H = L + F * cost / size with

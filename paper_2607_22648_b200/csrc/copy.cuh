@@ -24,7 +24,8 @@ struct Paged {                 // device view of ptstore_paged_cache_t
   u64 kv_stride, block_stride;
   u32 num_blocks;
   // COPY_FETCH_MULTI only: destination lists, one per distinct source block
-  const u32* head = nullptr;   // head[block id] = first node of the list, LINK_NIL if none
+  const u64* head = nullptr;   // low half of head[block id] = first node of the block's list (the block is in the
+                               // descriptor list, so the head was written by this call)
   const int2* node = nullptr;  // node[e] = {next node or LINK_NIL, cache block}
 };
 
@@ -33,7 +34,6 @@ struct Paged {                 // device view of ptstore_paged_cache_t
 // DISTINCT source block; a piece is read once and written to every destination of the block's list, which
 // removes the repeated reads from DRAM (on the bench workload only ~40 % of the fetched blocks are distinct).
 enum CopyMode { COPY_FETCH = 0, COPY_INSERT = 1, COPY_POOL = 2, COPY_FETCH_MULTI = 3 };
-constexpr u32 LINK_NIL = 0xFFFFFFFFu;
 
 __device__ __forceinline__ unsigned char* cache_addr(const Paged& pc, u32 ls, u32 cache_block, u64 off) {
   return pc.layer_base[ls >> 1] + (u64)(ls & 1) * pc.kv_stride + (u64)cache_block * pc.block_stride + off;
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(THREADS) copy_vector_kernel(Store st, Paged pc
       if (o < left) v[k] = ld_stream(src + o);
     }
     if (MODE == COPY_FETCH_MULTI) {
-      u32 e = pc.head[d.x];
+      u32 e = (u32)pc.head[d.x];
       for (u32 guard = 0; e != LINK_NIL && guard < 0x7FFFFFFFu; ++guard) {      // every thread walks the same list
         const int2 nd = pc.node[e];
         unsigned char* to = cache_addr(pc, ls, (u32)nd.y, off);
@@ -131,8 +131,17 @@ __device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// bounded wait: gives up after `limit` polls and reports false
+__device__ __forceinline__ bool mbar_test_wait(u64* bar, u32 parity) {
+  u32 ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: gives up after `limit` polls and reports false.  A poll may suspend the thread for a short,
+// hardware-defined time; a limit of 1 is a single test that does not suspend at all.
 __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, u32 limit) {
+  if (limit <= 1) return mbar_test_wait(bar, parity);
   for (u32 i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
@@ -158,6 +167,7 @@ struct BulkTune {
   int stage_bytes;   // bytes per stage (multiple of 16)
   int group;         // consecutive pieces a CTA takes before striding to its next group
   int hint;          // 1: mark loads and stores evict-first in L2
+  u32 wait_limit;    // polls per wait for a load in the main loop before the CTA gives up (draining keeps BULK_POLL_LIMIT)
 };
 
 __device__ __forceinline__ u64 l2_evict_first_policy() {
@@ -260,7 +270,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(Store st, Paged pc, const
     if (tune.hint) bulk_g2s_hint(smem + (size_t)s * SB, src, bytes, &bars[s], policy);
     else bulk_g2s(smem + (size_t)s * SB, src, bytes, &bars[s]);
     if (MODE == COPY_FETCH_MULTI) {              // resolve destinations while the load flies
-      u32 e = pc.head[d.x];
+      u32 e = (u32)pc.head[d.x];
       u32 n = 0;
       while (e != LINK_NIL && n < (u32)BULK_DST_CACHE) {
         const int2 nd = pc.node[e];
@@ -280,7 +290,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(Store st, Paged pc, const
   u32 parity = 0;
   u64 i = 0;
   for (; i < mine; ++i) {
-    if (!mbar_wait_bounded(&bars[s], parity, BULK_POLL_LIMIT)) { ok = false; break; }
+    if (!mbar_wait_bounded(&bars[s], parity, tune.wait_limit)) { ok = false; break; }
     const u32 bytes = s_bytes[s];
     if (bytes) {
       if (MODE == COPY_FETCH_MULTI) {
@@ -363,7 +373,7 @@ __global__ void __launch_bounds__(32) copy_bulk_multi_kernel(Store st, Paged pc,
     rec = rec + 1 == (u32)MULTI_NREC ? 0 : rec + 1;
     const u32 id = (u32)desc[pair].x;
     rec_src[rec] = block_ptr(st, id);
-    u32 e = pc.head[id], n = 0;
+    u32 e = (u32)pc.head[id], n = 0;
     while (e != LINK_NIL && n < (u32)MULTI_KMAX) {
       const int2 nd = pc.node[e];
       rec_dst[rec][n++] = (u32)nd.y;
@@ -396,7 +406,7 @@ __global__ void __launch_bounds__(32) copy_bulk_multi_kernel(Store st, Paged pc,
   u32 parity = 0;
   bool ok = true;
   while (stored < issued) {
-    if (!mbar_wait_bounded(&bars[s], parity, BULK_POLL_LIMIT)) { ok = false; break; }
+    if (!mbar_wait_bounded(&bars[s], parity, tune.wait_limit)) { ok = false; break; }
     const u32 r = s_rec[s], lsx = s_ls[s], off = s_off[s], bytes = s_bytes[s];
     unsigned char* base = pc.layer_base[lsx >> 1] + (u64)(lsx & 1) * pc.kv_stride + off;
     const unsigned char* from = smem + (size_t)s * SB;
@@ -483,70 +493,6 @@ __global__ void __launch_bounds__(256) build_pairs_kernel(Store st, const int* _
   cnt0 = __reduce_add_sync(FULL, cnt0);
   cnt1 = __reduce_add_sync(FULL, cnt1);
   if ((threadIdx.x & 31) == 0) {
-    if (cnt0) atomicAdd(&st.ctrl->blocks_fetched[0], (u64)cnt0);
-    if (cnt1) atomicAdd(&st.ctrl->blocks_fetched[1], (u64)cnt1);
-  }
-}
-
-// ---- destination lists for COPY_FETCH_MULTI ---------------------------------------------------------------------
-__global__ void __launch_bounds__(256) fetch_begin_kernel(Store st, u32* __restrict__ head, u32 n_blocks) {
-  for (u32 i = blockIdx.x * blockDim.x + threadIdx.x; i < n_blocks; i += gridDim.x * blockDim.x) head[i] = LINK_NIL;
-  if (blockIdx.x == 0 && threadIdx.x == 0) { st.ctrl->n_pairs = 0; st.ctrl->n_pairs_host = 0; st.ctrl->work_counter = 0; }
-}
-
-// every (r, j < matched[r]) entry pushes {cache block} on the list of its source block; the entry that finds the
-// list empty also appends the block to a descriptor list (one descriptor per distinct source block): HBM-tier
-// sources go to `desc`, host-tier sources to `desc_host`, so that each tier gets the copy engine and the grid
-// that suit it (HBM bandwidth needs every SM, the host link is saturated by a few CTAs)
-__global__ void __launch_bounds__(256) fetch_link_kernel(Store st, const int* __restrict__ ids, const int* __restrict__ matched,
-                                                         const int* __restrict__ bt, int R, int max_blocks, u32 cache_blocks,
-                                                         u32* __restrict__ head, int2* __restrict__ node, int2* __restrict__ desc,
-                                                         int2* __restrict__ desc_host) {
-  const long long total = (long long)R * max_blocks;
-  const long long rounded = (total + 31) & ~31ll;
-  const int lane = threadIdx.x & 31;
-  u32 cnt0 = 0, cnt1 = 0;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < rounded; e += (long long)gridDim.x * blockDim.x) {
-    bool first = false;
-    int id = -1;
-    if (e < total) {
-      const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
-      int mr = matched[r];
-      mr = mr > max_blocks ? max_blocks : mr;
-      if (j < mr) {
-        id = ids[e];
-        const int cb = bt[e];
-        if (id < 0 || (u32)id >= st.n[0] + st.n[1] || cb < 0 || (u32)cb >= cache_blocks) {
-          raise(st, S_BOUNDS);
-          id = -1;
-        } else {
-          const u32 old = atomicExch(&head[id], (u32)e);
-          node[e] = make_int2((int)old, cb);
-          first = old == LINK_NIL;
-          if ((u32)id < st.n[0]) ++cnt0; else ++cnt1;
-        }
-      }
-    }
-    const bool on_host = first && (u32)id >= st.n[0];
-    const unsigned m = __ballot_sync(FULL, first && !on_host);
-    const unsigned mh = __ballot_sync(FULL, on_host);
-    if (m) {
-      u32 base = 0;
-      if (lane == __ffs(m) - 1) base = atomicAdd(&st.ctrl->n_pairs, (u32)__popc(m));
-      base = __shfl_sync(FULL, base, __ffs(m) - 1);
-      if (first && !on_host) desc[base + __popc(m & ((1u << lane) - 1u))] = make_int2(id, 0);
-    }
-    if (mh) {
-      u32 base = 0;
-      if (lane == __ffs(mh) - 1) base = atomicAdd(&st.ctrl->n_pairs_host, (u32)__popc(mh));
-      base = __shfl_sync(FULL, base, __ffs(mh) - 1);
-      if (on_host) desc_host[base + __popc(mh & ((1u << lane) - 1u))] = make_int2(id, 0);
-    }
-    if ((m | mh) && lane == 0) atomicAdd(&st.ctrl->blocks_fetched_distinct, (u64)(__popc(m) + __popc(mh)));
-  }
-  cnt0 = __reduce_add_sync(FULL, cnt0);
-  cnt1 = __reduce_add_sync(FULL, cnt1);
-  if (lane == 0) {
     if (cnt0) atomicAdd(&st.ctrl->blocks_fetched[0], (u64)cnt0);
     if (cnt1) atomicAdd(&st.ctrl->blocks_fetched[1], (u64)cnt1);
   }

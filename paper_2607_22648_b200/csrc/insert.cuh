@@ -1,49 +1,32 @@
 // Scatter-insert of new blocks (store operation: only the increment after the longest common prefix
 // is saved and appended to the trie, paper Section 4 summary paragraph and Section 4.1).
 //
-// The batch must behave as if requests were inserted one after the other in index order.  Phases
-// (one kernel each, all over the R*max_blocks elements e = (request r, block j)):
+// The batch must behave as if requests were inserted one after the other in index order.  All the
+// metadata work of a call runs in ONE cooperative kernel whose phases are separated by grid-wide
+// barriers (elements e = (request r, block j), R*max_blocks of them):
+//   rebuild : only when deleted table markers have piled up: move the table aside, clear it, put the
+//             live entries back.
+//   hash    : chained block keys (content hashes first, by one thread per block, when requests are few
+//             and long), and in the same sweep
 //   claim   : find the key of e in the table or claim an empty slot for it (atomicCAS on the key);
 //             every element that lands on a slot claimed in this call lowers slot.aux to its request
 //             index (atomicMin), so the lowest request presenting a new prefix becomes its creator.
-//   count   : flag(e) = "e creates a node"; per-CTA sums.
-//   plan    : scan of the CTA sums; grants = min(new nodes, free HBM blocks); ring head moves.
-//   assign  : rank(e) among creators in (r, j) order; rank < grants gets ring[head + rank], writes the
-//             slot value and the node's metadata and a copy descriptor; the others delete their claim.
+//   count   : flag(e) = "e creates a node"; sums per tile of 1024 elements.
+//   assign  : every CTA derives the allocation plan from the tile sums (grants = min(new nodes, free HBM
+//             blocks)); rank(e) among creators in (r, j) order; rank < grants gets ring[head + rank],
+//             writes the slot value, the node's metadata and a copy descriptor; the others delete
+//             their claim.
 //   finish  : every element reads its slot's block id (or -1) and refreshes the LRU stamp.
 // Ranking creators in (r, j) order and granting the first `free` of them equals the sequential rule:
 // a denied node's descendants always rank higher, so denials are prefix-closed per request.
 #pragma once
 #include "common.cuh"
+#include "lookup.cuh"
+#include "evict.cuh"
 
 namespace pts {
 
 constexpr int INS_THREADS = 1024;
-
-__global__ void __launch_bounds__(256) insert_claim_kernel(Store st, const u64* __restrict__ keys, int R, int max_blocks,
-                                                           u32* __restrict__ eslot, int* __restrict__ new_blocks) {
-  const long long total = (long long)R * max_blocks;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-    const u32 r = (u32)(e / max_blocks);
-    if (e % max_blocks == 0) new_blocks[r] = 0;
-    const u64 key = keys[e];
-    if (key == 0) { eslot[e] = NO_SLOT; continue; }
-    u64 s = home_slot(key, st.slots);
-    u32 got = NO_SLOT;
-    for (u64 i = 0; i < st.slots; ++i) {
-      u64 k = *reinterpret_cast<volatile u64*>(&st.table[s].key);
-      if (k == KEY_EMPTY) {
-        k = atomicCAS(&st.table[s].key, KEY_EMPTY, key);
-        if (k == KEY_EMPTY) k = key;                     // claimed
-      }
-      if (k == key) { got = (u32)s; break; }
-      s = (s + 1 == st.slots) ? 0 : s + 1;
-    }
-    eslot[e] = got;
-    if (got == NO_SLOT) { raise(st, S_TABLE_FULL); continue; }
-    if (*reinterpret_cast<volatile u32*>(&st.table[got].id) == NO_ID) atomicMin(&st.table[got].aux, r);
-  }
-}
 
 __device__ __forceinline__ u32 creator_flag(const Store& st, const u32* __restrict__ eslot, long long e, int max_blocks) {
   const u32 s = eslot[e];
@@ -66,106 +49,190 @@ __device__ __forceinline__ u32 block_scan_incl(u32 x, u32* warp_sums, u32* total
   __syncthreads();
   const u32 incl = x + (wid ? warp_sums[wid - 1] : 0);
   *total = warp_sums[31];
+  __syncthreads();                       // warp_sums may be reused by the caller's next scan
   return incl;
 }
 
-__global__ void __launch_bounds__(INS_THREADS) insert_count_kernel(Store st, const u32* __restrict__ eslot, long long total,
-                                                                   int max_blocks, u32* __restrict__ cta_sums) {
-  __shared__ u32 warp_sums[32];
-  const long long e = (long long)blockIdx.x * INS_THREADS + threadIdx.x;
-  const u32 f = e < total ? creator_flag(st, eslot, e, max_blocks) : 0;
-  u32 sum;
-  block_scan_incl(f, warp_sums, &sum);
-  if (threadIdx.x == 0) cta_sums[blockIdx.x] = sum;
+// find `key` or claim an empty slot for it; the lowest request index presenting a key claimed in this call owns it
+__device__ __forceinline__ u32 claim_slot(const Store& st, u64 key, u32 r) {
+  u64 s = home_slot(key, st.slots);
+  u32 got = NO_SLOT;
+  for (u64 i = 0; i < st.slots; ++i) {
+    u64 k = *reinterpret_cast<volatile u64*>(&st.table[s].key);
+    if (k == KEY_EMPTY) {
+      k = atomicCAS(&st.table[s].key, KEY_EMPTY, key);
+      if (k == KEY_EMPTY) k = key;                     // claimed
+    }
+    if (k == key) { got = (u32)s; break; }
+    s = (s + 1 == st.slots) ? 0 : s + 1;
+  }
+  if (got == NO_SLOT) { raise(st, S_TABLE_FULL); return got; }
+  if (*reinterpret_cast<volatile u32*>(&st.table[got].id) == NO_ID) atomicMin(&st.table[got].aux, r);
+  return got;
 }
 
-// single CTA: exclusive scan of cta_sums in place, then the allocation plan
-__global__ void __launch_bounds__(INS_THREADS) insert_plan_kernel(Store st, u32* __restrict__ cta_sums, u32 n_ctas, u32 rebuild_threshold) {
+struct InsertArgs {
+  const int* tokens;
+  const long long* offsets;
+  int R, max_blocks;
+  int split;                // 1: content hashes first, one thread per block (few long requests); needs L == 32
+  u64* keys;                // scratch [R*max_blocks]
+  u32* eslot;               // scratch [R*max_blocks]
+  u32* cta_sums;            // scratch [tiles]
+  const int* bt;            // block tables of the source cache, or null (metadata only)
+  u32 cache_blocks;
+  u64 epoch;
+  int2* desc;               // out: copy descriptors {pool block, cache block}, ctrl->n_pairs of them
+  int* ids_out;
+  int* new_blocks;
+  Slot* stash;
+  u32 rebuild_threshold;
+  u32 launch_seq;
+};
+
+template <int L>
+__global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArgs a) {
   __shared__ u32 warp_sums[32];
-  __shared__ u32 carry;
-  if (threadIdx.x == 0) carry = 0;
-  __syncthreads();
-  for (u32 base = 0; base < n_ctas; base += INS_THREADS) {
-    const u32 i = base + threadIdx.x;
-    const u32 x = i < n_ctas ? cta_sums[i] : 0;
-    u32 tile_total;
-    const u32 incl = block_scan_incl(x, warp_sums, &tile_total);
-    if (i < n_ctas) cta_sums[i] = carry + incl - x;
-    __syncthreads();
-    if (threadIdx.x == 0) carry += tile_total;
-    __syncthreads();
+  constexpr int G = 32 / L;
+  Ctrl* c = st.ctrl;
+  GridBarrier bar;
+  bar.init(c, a.launch_seq);
+  const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
+  const long long total = (long long)a.R * a.max_blocks;
+  const int max_blocks = a.max_blocks;
+  // plan inputs, read before anything in this launch changes them
+  const u32 head0 = c->ring[0].head, count0 = c->ring[0].count, tomb0 = c->tombstones;
+  const u64 inflation = st.policy ? c->inflation : 0;
+  const long long gthreads = (long long)gridDim.x * INS_THREADS;
+  const long long gtid = (long long)blockIdx.x * INS_THREADS + threadIdx.x;
+
+  const bool rebuild = tomb0 > a.rebuild_threshold;
+  if (rebuild) table_rebuild_coop(st, a.stash, bar);
+
+  // ---- hash + claim ----------------------------------------------------------------------------------------------------
+  if (a.split) {
+    for (long long e = gtid; e < total; e += gthreads) {
+      const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
+      if (j < full_blocks(a.offsets, r, st.block_tokens, max_blocks))
+        a.keys[e] = content_block(a.tokens + a.offsets[r] + (long long)j * st.block_tokens, st.block_tokens);
+    }
+    bar.sync(st);
   }
-  if (threadIdx.x == 0) {
-    Ctrl* c = st.ctrl;
-    if (c->tombstones > rebuild_threshold) { c->tombstones = 0; c->rebuilds += 1; }   // this call began with a rebuild
-    const u32 total_new = carry;
-    const u32 granted = total_new < c->ring[0].count ? total_new : c->ring[0].count;
+  {
+    const long long warps = gthreads >> 5, warp0 = gtid >> 5;
+    const long long groups = ((long long)a.R + G - 1) / G;
+    for (long long grp = warp0; grp < groups && bar.ok; grp += warps) {
+      const long long r = grp * G + sub;
+      const bool valid = r < a.R;
+      const int nblk = valid ? full_blocks(a.offsets, (int)r, st.block_tokens, max_blocks) : 0;
+      const long long tok0 = valid ? a.offsets[r] : 0;
+      u64 parent = st.root_key;
+      const int most = __reduce_max_sync(FULL, nblk);
+      for (int base = 0; base < most; base += L) {
+        const int j = base + sl;
+        const bool active = j < nblk;
+        u64 cc = 0;
+        if (active) cc = a.split ? a.keys[r * max_blocks + j] : content_block(a.tokens + tok0 + (long long)j * st.block_tokens, st.block_tokens);
+        const int steps = most - base < L ? most - base : L;
+        const u64 key = chain_chunk<L>(parent, cc, lane, steps);
+        if (active) {
+          a.keys[r * max_blocks + j] = key;
+          a.eslot[r * max_blocks + j] = claim_slot(st, key, (u32)r);
+        }
+        parent = __shfl_sync(FULL, key, (lane & ~(L - 1)) + L - 1);
+      }
+      if (valid) {
+        for (int j = nblk + sl; j < max_blocks; j += L) { a.keys[r * max_blocks + j] = 0; a.eslot[r * max_blocks + j] = NO_SLOT; }
+        if (sl == 0) a.new_blocks[r] = 0;
+      }
+    }
+  }
+  bar.sync(st);
+
+  // ---- count -----------------------------------------------------------------------------------------------------------
+  const long long n_tiles = (total + INS_THREADS - 1) / INS_THREADS;
+  for (long long t = blockIdx.x; t < n_tiles && bar.ok; t += gridDim.x) {
+    const long long e = t * INS_THREADS + threadIdx.x;
+    const u32 f = e < total ? creator_flag(st, a.eslot, e, max_blocks) : 0;
+    u32 sum;
+    block_scan_incl(f, warp_sums, &sum);
+    if (threadIdx.x == 0) a.cta_sums[t] = sum;
+  }
+  bar.sync(st);
+
+  // ---- plan (the same in every CTA) and assign -------------------------------------------------------------------------
+  u32 total_new;
+  {
+    u32 part = 0;
+    for (long long i = threadIdx.x; i < n_tiles; i += INS_THREADS) part += a.cta_sums[i];
+    block_scan_incl(part, warp_sums, &total_new);
+  }
+  const u32 granted = total_new < count0 ? total_new : count0;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && bar.ok) {
+    if (rebuild) c->rebuilds += 1;
     c->ins_total_new = total_new;
     c->ins_granted = granted;
-    c->ins_base = c->ring[0].head;
-    c->ring[0].head = (u32)(((u64)c->ring[0].head + granted) % st.n[0]);
-    c->ring[0].count -= granted;
+    c->ins_base = head0;
+    c->ring[0].head = (u32)(((u64)head0 + granted) % st.n[0]);
+    c->ring[0].count = count0 - granted;
     c->live[0] += granted;
     c->n_pairs = granted;
     c->blocks_inserted += granted;
     c->blocks_denied += total_new - granted;
-    c->tombstones += total_new - granted;
+    c->tombstones = (rebuild ? 0 : tomb0) + (total_new - granted);
     if (granted < total_new) atomicOr(&c->status, S_NOSPACE);
   }
-}
-
-__global__ void __launch_bounds__(INS_THREADS) insert_assign_kernel(Store st, const u64* __restrict__ keys,
-                                                                    const u32* __restrict__ eslot, long long total, int max_blocks,
-                                                                    const u32* __restrict__ cta_sums, const int* __restrict__ bt,
-                                                                    u32 cache_blocks, u64 epoch, int2* __restrict__ desc,
-                                                                    int* __restrict__ new_blocks) {
-  __shared__ u32 warp_sums[32];
-  const long long e = (long long)blockIdx.x * INS_THREADS + threadIdx.x;
-  const u32 f = e < total ? creator_flag(st, eslot, e, max_blocks) : 0;
-  u32 sum;
-  const u32 incl = block_scan_incl(f, warp_sums, &sum);
-  if (!f) return;
-  const u32 rank = cta_sums[blockIdx.x] + incl - 1;
-  const u32 granted = st.ctrl->ins_granted;
-  Slot* slot = st.table + eslot[e];
-  if (rank >= granted) {                       // denied: withdraw the claim
+  for (long long t = blockIdx.x; t < n_tiles && bar.ok; t += gridDim.x) {
+    u32 before;                                   // creators in earlier tiles
+    {
+      u32 part = 0;
+      for (long long i = threadIdx.x; i < t; i += INS_THREADS) part += a.cta_sums[i];
+      block_scan_incl(part, warp_sums, &before);
+    }
+    const long long e = t * INS_THREADS + threadIdx.x;
+    const u32 f = e < total ? creator_flag(st, a.eslot, e, max_blocks) : 0;
+    u32 sum;
+    const u32 incl = block_scan_incl(f, warp_sums, &sum);
+    if (!f) continue;
+    const u32 rank = before + incl - 1;
+    Slot* slot = st.table + a.eslot[e];
+    if (rank >= granted) {                       // denied: withdraw the claim
+      slot->aux = NO_ID;
+      slot->key = KEY_TOMB;
+      continue;
+    }
+    const u32 id = (u32)st.ring_ids[0][(u32)(((u64)head0 + rank) % st.n[0])];
+    const int j = (int)(e % max_blocks);
+    st.m_key[id] = a.keys[e];
+    st.m_parent[id] = j ? a.keys[e - 1] : st.root_key;
+    st.m_last[id] = st.policy ? 0 : a.epoch;    // GDSF: the finish phase counts this call's accesses
+    st.m_freq[id] = 0;
+    st.m_ref[id] = 0;
+    st.m_depth[id] = (u32)j;
     slot->aux = NO_ID;
-    slot->key = KEY_TOMB;
-    return;
+    slot->id = id;
+    int2 d = make_int2((int)id, 0);
+    if (a.bt) {
+      const int cb = a.bt[e];
+      if (cb < 0 || (u32)cb >= a.cache_blocks) { raise(st, S_BOUNDS); d.x = -1; }
+      d.y = cb;
+    } else {
+      d.x = -1;                                  // metadata-only insert: nothing to copy
+    }
+    a.desc[rank] = d;
+    atomicAdd(&a.new_blocks[e / max_blocks], 1);
   }
-  const u32 id = (u32)st.ring_ids[0][(u32)(((u64)st.ctrl->ins_base + rank) % st.n[0])];
-  const int j = (int)(e % max_blocks);
-  st.m_key[id] = keys[e];
-  st.m_parent[id] = j ? keys[e - 1] : st.root_key;
-  st.m_last[id] = st.policy ? 0 : epoch;      // GDSF: the finish kernel counts this call's accesses
-  st.m_freq[id] = 0;
-  st.m_ref[id] = 0;
-  st.m_depth[id] = (u32)j;
-  slot->aux = NO_ID;
-  slot->id = id;
-  int2 d = make_int2((int)id, 0);
-  if (bt) {
-    const int cb = bt[e];
-    if (cb < 0 || (u32)cb >= cache_blocks) { raise(st, S_BOUNDS); d.x = -1; }
-    d.y = cb;
-  } else {
-    d.x = -1;                                  // metadata-only insert: nothing to copy
-  }
-  desc[rank] = d;
-  atomicAdd(&new_blocks[e / max_blocks], 1);
-}
+  bar.sync(st);
 
-__global__ void __launch_bounds__(256) insert_finish_kernel(Store st, const u32* __restrict__ eslot, long long total, u64 epoch,
-                                                            int* __restrict__ ids_out) {
-  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-    const u32 s = eslot[e];
+  // ---- finish ----------------------------------------------------------------------------------------------------------
+  for (long long e = gtid; e < total && bar.ok; e += gthreads) {
+    const u32 s = a.eslot[e];
     int out = -1;
     if (s != NO_SLOT) {
       const u32 id = st.table[s].id;
-      if (id != NO_ID) { out = (int)id; touch_block(st, id, epoch, inflation, 1); }
+      if (id != NO_ID) { out = (int)id; touch_block(st, id, a.epoch, inflation, 1); }
     }
-    ids_out[e] = out;
+    a.ids_out[e] = out;
   }
 }
 

@@ -34,6 +34,69 @@ __device__ __forceinline__ u64 chain_chunk(u64& parent, u64 c, int lane, int ste
   return mine;
 }
 
+// ---- destination lists of a fetch --------------------------------------------------------------------------------
+// A batch of prompts over popular documents names the same pool block many times (a block is a trie node, so equal
+// ids always sit at the same depth of different requests).  A fetch therefore reads each DISTINCT source block once
+// and writes it to every destination: each (request, block) entry pushes its cache block on the list of its source
+// block, and the entry that finds the list empty appends the block to a descriptor list (HBM-tier sources and
+// host-tier sources separately, so that each gets the copy engine and the grid that suit it).  List heads carry the
+// sequence number of the fetch call in their upper half: a head written by an earlier call reads as "empty", so
+// nothing has to be cleared between calls.
+struct FetchLink {
+  const int* bt;        // block tables of the destination cache; null = no fetch attached to this lookup
+  u32 cache_blocks;
+  u32 seq;              // sequence number of this fetch call (never 0)
+  u32 pending_seq;      // tag of a demotion copy still running on the side stream, 0 if none
+  u64* heads;           // [block id] = seq << 32 | entry index of the first list node
+  int2* node;           // [entry] = {next entry or LINK_NIL, cache block}
+  int2* desc;           // distinct HBM-tier source blocks
+  int2* desc_host;      // distinct host-tier source blocks
+};
+
+// one entry: returns 1 if it opened the list of an HBM-tier block, 2 for a host-tier block, 0 otherwise
+__device__ __forceinline__ int link_entry(const Store& st, const FetchLink& fl, long long e, int id, u32& cnt0, u32& cnt1) {
+  const int cb = fl.bt[e];
+  if (id < 0 || (u32)id >= st.n[0] + st.n[1] || cb < 0 || (u32)cb >= fl.cache_blocks) { raise(st, S_BOUNDS); return 0; }
+  if (fl.pending_seq && (u32)id >= st.n[0] && st.m_flight[id] == fl.pending_seq) { raise(st, S_INFLIGHT); return 0; }
+  const u64 old = atomicExch(&fl.heads[id], ((u64)fl.seq << 32) | (u64)(u32)e);
+  const bool fresh = (u32)(old >> 32) != fl.seq;
+  fl.node[e] = make_int2(fresh ? (int)LINK_NIL : (int)(u32)old, cb);
+  if ((u32)id < st.n[0]) ++cnt0; else ++cnt1;
+  return fresh ? ((u32)id < st.n[0] ? 1 : 2) : 0;
+}
+// all 32 lanes: append the blocks whose lists were opened to the descriptor lists (one atomic per warp and list)
+__device__ __forceinline__ void link_append(const Store& st, const FetchLink& fl, int opened, int id, int lane) {
+  const unsigned m = __ballot_sync(FULL, opened == 1);
+  const unsigned mh = __ballot_sync(FULL, opened == 2);
+  const u32 slot = fl.seq & 1u;
+  if (m) {
+    u32 base = 0;
+    if (lane == __ffs(m) - 1) base = atomicAdd(&st.ctrl->f_pairs[slot], (u32)__popc(m));
+    base = __shfl_sync(FULL, base, __ffs(m) - 1);
+    if (opened == 1) fl.desc[base + __popc(m & ((1u << lane) - 1u))] = make_int2(id, 0);
+  }
+  if (mh) {
+    u32 base = 0;
+    if (lane == __ffs(mh) - 1) base = atomicAdd(&st.ctrl->f_pairs_host[slot], (u32)__popc(mh));
+    base = __shfl_sync(FULL, base, __ffs(mh) - 1);
+    if (opened == 2) fl.desc_host[base + __popc(mh & ((1u << lane) - 1u))] = make_int2(id, 0);
+  }
+  if ((m | mh) && lane == 0) atomicAdd(&st.ctrl->blocks_fetched_distinct, (u64)(__popc(m) + __popc(mh)));
+}
+// once per linking kernel: clear the per-call scalars of the NEXT fetch call
+__device__ __forceinline__ void link_prepare_next(const Store& st, const FetchLink& fl) {
+  const u32 nxt = (fl.seq & 1u) ^ 1u;
+  st.ctrl->f_pairs[nxt] = 0; st.ctrl->f_pairs_host[nxt] = 0; st.ctrl->f_work[nxt] = 0;
+}
+__device__ __forceinline__ void link_count(const Store& st, u32 cnt0, u32 cnt1, int lane) {
+  cnt0 = __reduce_add_sync(FULL, cnt0);
+  cnt1 = __reduce_add_sync(FULL, cnt1);
+  if (lane == 0) {
+    if (cnt0) atomicAdd(&st.ctrl->blocks_fetched[0], (u64)cnt0);
+    if (cnt1) atomicAdd(&st.ctrl->blocks_fetched[1], (u64)cnt1);
+  }
+}
+
 // keys_out[r*max_blocks + j] = chained key of block j, 0 beyond the request's full blocks
 template <int L>
 __global__ void __launch_bounds__(256) hash_kernel(Store st, const int* __restrict__ tokens,
@@ -65,7 +128,7 @@ template <int L>
 __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __restrict__ tokens,
                                                      const long long* __restrict__ offsets, int R, int max_blocks,
                                                      u32 flags, u64 epoch, int* __restrict__ matched,
-                                                     int* __restrict__ ids_out) {
+                                                     int* __restrict__ ids_out, FetchLink fl) {
   constexpr int G = 32 / L;
   constexpr unsigned SUBMASK = (L == 32) ? FULL : ((1u << L) - 1u);
   const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
@@ -79,6 +142,8 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
   int m = 0;
   bool done = nblk == 0;
   u32 my_probes = 0, my_visited = 0;
+  u32 cnt0 = 0, cnt1 = 0;
+  if (fl.bt && blockIdx.x == 0 && threadIdx.x == 0) link_prepare_next(st, fl);
 
   for (int base = 0;; base += L) {
     const unsigned going = __ballot_sync(FULL, !done);
@@ -123,12 +188,17 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
         }
       }
     }
+    if (fl.bt) {                                                 // fetch attached: link the hits to their source blocks
+      const int opened = hit ? link_entry(st, fl, r * max_blocks + j, (int)id, cnt0, cnt1) : 0;
+      link_append(st, fl, opened, (int)id, lane);
+    }
     if (!done) {
       m += nf;
       if (nf < L || base + L >= nblk) done = true;
     }
     parent = __shfl_sync(FULL, key, (lane & ~(L - 1)) + L - 1);
   }
+  if (fl.bt) link_count(st, cnt0, cnt1, lane);
 
   if (valid) {
     for (int j = m + sl; j < max_blocks; j += L) ids_out[r * max_blocks + j] = -1;
@@ -186,11 +256,13 @@ __global__ void __launch_bounds__(128) chain_kernel(Store st, const u64* content
 
 __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* __restrict__ content, const long long* __restrict__ offsets,
                                                            int R, int max_blocks, u32 flags, u64 epoch, int* __restrict__ matched,
-                                                           int* __restrict__ ids_out) {
+                                                           int* __restrict__ ids_out, FetchLink fl) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long r = warp;
+  if (fl.bt && blockIdx.x == 0 && threadIdx.x == 0) link_prepare_next(st, fl);
   if (r >= R) return;
+  u32 cnt0 = 0, cnt1 = 0;
   const int nblk = full_blocks(offsets, (int)r, st.block_tokens, max_blocks);
   const u64 inflation = st.policy ? st.ctrl->inflation : 0;
   const u64* crow = content + r * max_blocks;
@@ -241,10 +313,15 @@ __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* 
         }
       }
     }
+    if (fl.bt) {
+      const int opened = hit ? link_entry(st, fl, r * max_blocks + j, (int)id, cnt0, cnt1) : 0;
+      link_append(st, fl, opened, (int)id, lane);
+    }
     m += nf;
     if (nf < 32) break;
     key = next_key;
   }
+  if (fl.bt) link_count(st, cnt0, cnt1, lane);
   for (int j = m + lane; j < max_blocks; j += 32) ids_out[r * max_blocks + j] = -1;
   if (lane == 0) matched[r] = m;
   u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
@@ -256,6 +333,30 @@ __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* 
     const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
     if (v) atomicAdd(&st.ctrl->lookup_stripes[warp % LOOKUP_STRIPES][lane], (u64)v);
   }
+}
+
+// the linking step on its own, for a fetch of ids the caller already holds: every (r, j < matched[r]) entry
+__global__ void __launch_bounds__(256) fetch_link_kernel(Store st, const int* __restrict__ ids, const int* __restrict__ matched, int R,
+                                                         int max_blocks, FetchLink fl) {
+  const long long total = (long long)R * max_blocks;
+  const long long rounded = (total + 31) & ~31ll;
+  const int lane = threadIdx.x & 31;
+  u32 cnt0 = 0, cnt1 = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) link_prepare_next(st, fl);
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < rounded; e += (long long)gridDim.x * blockDim.x) {
+    int opened = 0, id = -1;
+    if (e < total) {
+      const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
+      int mr = matched[r];
+      mr = mr > max_blocks ? max_blocks : mr;
+      if (j < mr) {
+        id = ids[e];
+        opened = link_entry(st, fl, e, id, cnt0, cnt1);
+      }
+    }
+    link_append(st, fl, opened, id, lane);
+  }
+  link_count(st, cnt0, cnt1, lane);
 }
 
 // refcount-- per (r, j < matched[r]) pair; a zero count stays zero and raises S_STATE

@@ -22,10 +22,14 @@ constexpr u64 ALIGN = 256;
 inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
-  u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, ring[2], ctrl, blocked, sort[2], hist, room, desc, keys, eslot,
-      cta_sums, prefix, promo_first, promo_cnt, links, desc_tier, desc_host, total;
-  u32 n_tiles;
+  u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, m_flight, ring[2], ctrl, blocked, sort[2], hist, tile_stats, room, desc,
+      keys, eslot, cta_sums, prefix, promo_first, promo_cnt, heads, links, desc_tier, desc_host, total;
 };
+
+constexpr u32 MAX_COOP_GRID = 256;      // cooperative kernels use at most this many CTAs (and at most one per SM)
+constexpr u64 MIN_SLOTS = 2 * PROBE_WINDOW;   // the windowed probe wraps an index once, so a table is never smaller than this
+
+inline u64 effective_slots(const ptstore_config_t* c) { return c->table_slots < MIN_SLOTS ? MIN_SLOTS : c->table_slots; }
 
 bool geometry_ok(const ptstore_config_t* c) {
   if (!c || c->struct_size != sizeof(ptstore_config_t)) return false;
@@ -41,20 +45,21 @@ bool geometry_ok(const ptstore_config_t* c) {
 
 Layout make_layout(const ptstore_config_t* c) {
   Layout L;
-  const u64 N = (u64)c->hbm_blocks + c->host_blocks, M = c->max_batch_blocks;
+  const u64 N = (u64)c->hbm_blocks + c->host_blocks, M = c->max_batch_blocks, S = effective_slots(c);
   u64 o = 0;
   auto take = [&](u64 bytes) { u64 at = o; o = align_up(o + (bytes ? bytes : 1)); return at; };
-  L.table[0] = take(c->table_slots * sizeof(Slot));
-  L.table[1] = take(c->table_slots * sizeof(Slot));
+  L.table[0] = take(S * sizeof(Slot));
+  L.table[1] = take(S * sizeof(Slot));
   L.m_key = take(N * 8); L.m_parent = take(N * 8); L.m_last = take(N * 8);
-  L.m_freq = take(N * 4); L.m_ref = take(N * 4); L.m_depth = take(N * 4);
+  L.m_freq = take(N * 4); L.m_ref = take(N * 4); L.m_depth = take(N * 4); L.m_flight = take(N * 4);
   L.ring[0] = take((u64)c->hbm_blocks * 4); L.ring[1] = take((u64)c->host_blocks * 4);
   L.ctrl = take(sizeof(Ctrl));
   L.blocked = take(N);
-  L.sort[0] = take(N * sizeof(Key2)); L.sort[1] = take(N * sizeof(Key2));
-  const u64 sort_tile = (u64)SORT_THREADS * sort_steps_for(N);
-  L.n_tiles = (u32)((N + sort_tile - 1) / sort_tile);
-  L.hist = take((u64)256 * L.n_tiles * 4);
+  // eviction: one sort record per block id of a tier, padded to whole tiles of the largest grid
+  const u64 recs = N + (u64)MAX_COOP_GRID * EV_THREADS;
+  L.sort[0] = take(recs * sizeof(Key2)); L.sort[1] = take(recs * sizeof(Key2));
+  L.hist = take((u64)256 * MAX_COOP_GRID * 4);
+  L.tile_stats = take((u64)MAX_COOP_GRID * 4 * 8);
   L.room = take((u64)c->host_blocks * 4);
   L.desc = take((M > N ? M : N) * sizeof(int2));
   L.keys = take(M * 8);
@@ -63,6 +68,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.prefix = take(((u64)c->max_requests + 1) * 4);
   L.promo_first = take(N * 4);
   L.promo_cnt = take(N * 4);
+  L.heads = take(N * 8);
   L.links = take(M * sizeof(int2));
   L.desc_tier = take((u64)c->hbm_blocks * sizeof(int2));
   L.desc_host = take((c->host_blocks ? (M < c->host_blocks ? M : (u64)c->host_blocks) : 1) * sizeof(int2));
@@ -82,6 +88,7 @@ struct ptstore {
   unsigned char* blocked;
   Key2* sort_buf[2];
   u32* hist;
+  u64* tile_stats;
   int* room;
   int2* desc;
   u64* keys;
@@ -90,21 +97,26 @@ struct ptstore {
   u32* prefix;
   u32* promo_first;
   u32* promo_cnt;
+  u64* heads;            // fetch: tagged heads of the destination lists, one per block id
   int2* links;           // fetch: destination list nodes, one per (request, block) entry
   int2* desc_tier;       // demotion: {HBM id, host id} pairs
   int2* desc_host;       // fetch: descriptors of distinct host-tier source blocks
   int host_ctas;         // grid of the copies that run at host-link speed
-  cudaStream_t tier_stream;   // side stream of ptstore_evict_async (created on first use)
+  cudaStream_t tier_stream;   // side stream of the asynchronous demotion copy (created on first use)
   cudaEvent_t ev_meta, ev_copy;
   bool tier_ready, tier_pending;
+  u32 flight_seq;        // tag of the demotion copy that may still be running (valid while tier_pending)
+  u32 fetch_seq;         // sequence number of the last fetch call (tags the list heads; never 0)
+  u32 coop_seq;          // cooperative launches so far (selects the barrier counter)
+  u32 wait_limit;        // polls per bounded wait in the copy kernels' main loop
+  cudaEvent_t time_before, time_after;   // one-shot: recorded around the next HBM copy kernel (ptstore_time_next_copy)
+  int coop_grid;         // CTAs a cooperative kernel may use: one per SM, at most MAX_COOP_GRID
   u64 epoch;
   u64 launches;
   int last_cuda;
   int sms;
   int bulk_smem_set[4];
   int bulk_multi_smem_set;  // dynamic shared memory already granted to the bulk kernel of each mode
-  bool has_env_tune;
-  BulkVariant env_tune;
 };
 
 namespace {
@@ -147,6 +159,17 @@ Paged to_paged(const ptstore_paged_cache_t* pc) {
   return p;
 }
 
+// a kernel whose CTAs wait for one another at grid-wide barriers: all of them must be resident at once
+template <typename Kernel, typename Args>
+int launch_coop(ptstore* h, Kernel kernel, int grid, int threads, Args& args, cudaStream_t s) {
+  args.launch_seq = ++h->coop_seq;
+  void* params[2] = {&h->st, &args};
+  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), params, 0, s);
+  h->launches += 1;
+  if (e != cudaSuccess) { (void)cudaGetLastError(); h->last_cuda = (int)e; return PTSTORE_E_CUDA; }
+  return PTSTORE_OK;
+}
+
 template <int L>
 int launch_hash(ptstore* h, const int* tokens, const long long* offsets, int R, int max_blocks, u64* keys, cudaStream_t s) {
   const long long warps = ((long long)R + (32 / L) - 1) / (32 / L);
@@ -157,10 +180,10 @@ int launch_hash(ptstore* h, const int* tokens, const long long* offsets, int R, 
 }
 template <int L>
 int launch_lookup(ptstore* h, const int* tokens, const long long* offsets, int R, int max_blocks, u32 flags, int* matched,
-                  int* ids, cudaStream_t s) {
+                  int* ids, const FetchLink& fl, cudaStream_t s) {
   const long long warps = ((long long)R + (32 / L) - 1) / (32 / L);
   const int grid = (int)((warps * 32 + 255) / 256);
-  lookup_kernel<L><<<grid, 256, 0, s>>>(h->st, tokens, offsets, R, max_blocks, flags, h->epoch, matched, ids);
+  lookup_kernel<L><<<grid, 256, 0, s>>>(h->st, tokens, offsets, R, max_blocks, flags, h->epoch, matched, ids, fl);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
@@ -197,39 +220,18 @@ int lanes_for(const ptstore* h, int R, int max_blocks) {
 }
 
 // ---- copy engine dispatch -----------------------------------------------------------------------------------
-// index = PTSTORE_COPY_VARIANT field of the flags
+// Ring geometries selectable with PTSTORE_COPY_VARIANT (see include/ptstore.h); 0 sizes the ring from the chunk size.
 const BulkVariant kBulkVariants[] = {
     {0, 0, 1, 1, 0},       // 0: default, sized by auto_bulk() from the chunk size
-    {8, 8192, 3, 1, 0},    // 1
-    {3, 32768, 1, 1, 0},   // 2
-    {4, 16384, 3, 1, 0},   // 3
-    {8, 16384, 1, 1, 0},   // 4
-    {12, 16384, 1, 1, 0},  // 5
-    {4, 32768, 1, 1, 0},   // 6
-    {6, 32768, 1, 1, 0},   // 7
-    {6, 16384, 1, 2, 0},   // 8: a CTA takes whole 32 KiB chunks
-    {6, 16384, 1, 1, 1},   // 9: evict-first L2 hints
-    {3, 65536, 1, 1, 0},   // 10
-    {24, 8192, 1, 1, 0},   // 11
+    {8, 8192, 3, 1, 0},    // 1: 8 stages of 8 KiB, 3 CTAs per SM
+    {3, 32768, 1, 1, 0},   // 2: 3 stages of 32 KiB
+    {4, 16384, 3, 1, 0},   // 3: 4 stages of 16 KiB, 3 CTAs per SM
+    {12, 16384, 1, 1, 0},  // 4: 12 stages of 16 KiB
+    {6, 16384, 1, 2, 0},   // 5: 6 stages of 16 KiB, a CTA takes two consecutive pieces at a time
+    {6, 16384, 1, 1, 1},   // 6: 6 stages of 16 KiB, loads and stores marked evict-first in L2
+    {3, 65536, 1, 1, 0},   // 7: 3 stages of 64 KiB
 };
 constexpr int kNumBulkVariants = (int)(sizeof(kBulkVariants) / sizeof(kBulkVariants[0]));
-
-// PTSTORE_BULK_TUNE="stages,stage_bytes,ctas_per_sm,group,hint" overrides the variant table (tuning aid)
-bool env_bulk_tune(BulkVariant* v) {
-  const char* e = std::getenv("PTSTORE_BULK_TUNE");
-  if (!e) return false;
-  int a[5] = {0, 0, 0, 1, 0};
-  int n = 0;
-  const char* p = e;
-  while (*p && n < 5) {
-    a[n++] = std::atoi(p);
-    while (*p && *p != ',') ++p;
-    if (*p == ',') ++p;
-  }
-  if (n < 3 || a[0] < 2 || a[0] > BULK_MAX_STAGES || a[1] < 16 || a[1] % 16 || (long long)a[0] * a[1] > 227 * 1024 || a[2] < 1 || a[3] < 1) return false;
-  *v = {a[0], a[1], a[2], a[3], a[4] ? 1 : 0};
-  return true;
-}
 
 // Default ring, from measurements on B200 (read+write GB/s of the fetch / insert copies on the bench workload):
 //   32 KiB chunks: 3 x 32 KiB x 1 CTA per SM 6.65 / 6.46 TB/s (deeper rings and more CTAs lose 3-7 %: few bytes in flight win)
@@ -245,7 +247,7 @@ BulkVariant auto_bulk(u64 chunk_bytes) {
 }
 
 template <int MODE>
-int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, const BulkVariant& v, int ctas_per_sm) {
+int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, const BulkVariant& v, int ctas_per_sm, const int2* desc, const u32* n_pairs) {
   const int smem = v.stages * v.stage_bytes;
   if (smem > h->bulk_smem_set[MODE]) {
     if (cudaFuncSetAttribute(copy_bulk_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -254,14 +256,15 @@ int launch_bulk(ptstore* h, const Paged& pc, cudaStream_t s, const BulkVariant& 
     }
     h->bulk_smem_set[MODE] = smem;
   }
-  BulkTune t = {v.stages, v.stage_bytes, v.group, v.hint};
-  copy_bulk_kernel<MODE><<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs, t);
+  BulkTune t = {v.stages, v.stage_bytes, v.group, v.hint, h->wait_limit};
+  copy_bulk_kernel<MODE><<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, desc, n_pairs, t);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
 
 // multi-destination fetch: dynamic dealing of `group`-piece units (default: a quarter of a source block)
-int launch_bulk_multi(ptstore* h, const Paged& pc, cudaStream_t s, BulkVariant v, int ctas_per_sm) {
+int launch_bulk_multi(ptstore* h, const Paged& pc, cudaStream_t s, BulkVariant v, int ctas_per_sm, const int2* desc, const u32* n_pairs,
+                      u32* work_counter) {
   const int smem = v.stages * v.stage_bytes;
   if (smem > h->bulk_multi_smem_set) {
     if (cudaFuncSetAttribute(copy_bulk_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -273,29 +276,37 @@ int launch_bulk_multi(ptstore* h, const Paged& pc, cudaStream_t s, BulkVariant v
   const u32 ppc = (u32)((h->st.chunk_bytes + v.stage_bytes - 1) / v.stage_bytes);
   const u32 per_pair = 2u * h->st.layers * ppc;
   int group = v.group > 1 ? v.group : (int)(per_pair >= 4 ? per_pair / 4 : per_pair);
-  BulkTune t = {v.stages, v.stage_bytes, group, 0};
-  copy_bulk_multi_kernel<<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, h->desc, &h->st.ctrl->n_pairs, &h->st.ctrl->work_counter, t);
+  BulkTune t = {v.stages, v.stage_bytes, group, 0, h->wait_limit};
+  copy_bulk_multi_kernel<<<h->sms * ctas_per_sm, 32, smem, s>>>(h->st, pc, desc, n_pairs, work_counter, t);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
 
+// desc / n_pairs: the descriptor list to copy; grid > 0: a copy at host-link speed (fixed small grid, vector engine)
 template <int MODE>
-int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream_t s, const int2* desc = nullptr,
-                const u32* n_pairs = nullptr, int grid = 0) {
-  if (!desc) { desc = h->desc; n_pairs = &h->st.ctrl->n_pairs; }
-  if (grid > 0) {       // host-link copies: fixed small grid, vector engine
+int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream_t s, const int2* desc, const u32* n_pairs, int grid = 0,
+                u32* work_counter = nullptr) {
+  if (grid > 0) {
     copy_vector_kernel<MODE, 256, 8><<<grid, 256, 0, s>>>(h->st, pc, desc, n_pairs);
     PTS_CHECK_LAUNCH(h);
     return PTSTORE_OK;
   }
+  // a caller who asked for it gets its two events recorded around this kernel (one shot)
+  struct Timer {
+    ptstore* h; cudaStream_t s; cudaEvent_t after;
+    Timer(ptstore* h_, cudaStream_t s_) : h(h_), s(s_), after(h_->time_after) {
+      if (h->time_before) cudaEventRecord(h->time_before, s);
+      h->time_before = nullptr; h->time_after = nullptr;
+    }
+    ~Timer() { if (after) cudaEventRecord(after, s); }
+  } timer(h, s);
   const u32 variant = (h->cfg.flags >> 16) & 0xFu;
   int per_sm = (int)((h->cfg.flags >> 20) & 0xFFu);
   if (!(h->cfg.flags & PTSTORE_COPY_VECTOR) && !host_side_possible) {
     BulkVariant v = kBulkVariants[variant < (u32)kNumBulkVariants ? variant : 0];
     if (v.stages == 0) v = auto_bulk(h->st.chunk_bytes);
-    if (h->has_env_tune) v = h->env_tune;
-    if (MODE == COPY_FETCH_MULTI && !v.hint) return launch_bulk_multi(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm);
-    return launch_bulk<MODE>(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm);
+    if (MODE == COPY_FETCH_MULTI && !v.hint) return launch_bulk_multi(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm, desc, n_pairs, work_counter);
+    return launch_bulk<MODE>(h, pc, s, v, per_sm ? per_sm : v.ctas_per_sm, desc, n_pairs);
   }
   switch (variant) {
     case 1:
@@ -312,87 +323,10 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
   return PTSTORE_OK;
 }
 
-// ---- radix sort of the eviction candidates ----------------------------------------------------------------------
-int bytes_needed(u64 max_value) {
-  int b = 0;
-  while (max_value) { ++b; max_value >>= 8; }
-  return b ? b : 1;
-}
-
-// sorts sort_buf[0][0..ev_cand) ; returns the index of the buffer that holds the result in *result
-int launch_sort(ptstore* h, cudaStream_t s, int* result) {
-  const u32 nt = h->lay.n_tiles;
-  const bool small = sort_steps_for((u64)h->cfg.hbm_blocks + h->cfg.host_blocks) == 2;
-  int cur = 0;
-  struct Pass { int word, shift; } passes[16];
-  int np = 0;
-  const int id_bytes = bytes_needed((u64)h->cfg.hbm_blocks + h->cfg.host_blocks - 1);
-  for (int b = 0; b < id_bytes; ++b) passes[np++] = {0, 8 * b};
-  passes[np++] = {0, 32};
-  passes[np++] = {0, 40};
-  // LRU: stamps are at most the epoch.  GDSF: a priority H = L + F has no bound the host knows (L accumulates the
-  // priorities of earlier victims), so the whole word is sorted
-  const int st_bytes = h->st.policy ? 8 : bytes_needed(h->epoch);
-  for (int b = 0; b < st_bytes; ++b) passes[np++] = {1, 8 * b};
-  for (int p = 0; p < np; ++p) {
-    if (small) sort_hist_kernel<2><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
-    else sort_hist_kernel<8><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], &h->st.ctrl->ev_cand, passes[p].word, passes[p].shift, h->hist, nt);
-    PTS_CHECK_LAUNCH(h);
-    sort_scan_kernel<<<1, 1024, 0, s>>>(h->hist, 256u * nt);
-    PTS_CHECK_LAUNCH(h);
-    if (small) sort_scatter_kernel<2><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], h->sort_buf[cur ^ 1], &h->st.ctrl->ev_cand, passes[p].word,
-                                                                passes[p].shift, h->hist, nt);
-    else sort_scatter_kernel<8><<<nt, SORT_THREADS, 0, s>>>(h->sort_buf[cur], h->sort_buf[cur ^ 1], &h->st.ctrl->ev_cand, passes[p].word,
-                                                     passes[p].shift, h->hist, nt);
-    PTS_CHECK_LAUNCH(h);
-    cur ^= 1;
-  }
-  *result = cur;
-  return PTSTORE_OK;
-}
-
 // deleted markers are reclaimed at the start of an insert once they exceed 1/8 of the table (device-side decision)
-inline u32 rebuild_threshold(const ptstore* h) { return (u32)(h->cfg.table_slots / 8); }
+inline u32 rebuild_threshold(const ptstore* h) { return (u32)(h->st.slots / 8); }
 
-int maybe_rebuild(ptstore* h, cudaStream_t s) {
-  const int cap = h->sms * 8;
-  table_stash_kernel<<<grid_for((long long)h->cfg.table_slots, 256, cap), 256, 0, s>>>(h->st, h->stash, rebuild_threshold(h));
-  PTS_CHECK_LAUNCH(h);
-  table_rebuild_kernel<<<grid_for((long long)h->cfg.table_slots, 256, cap), 256, 0, s>>>(h->st, h->stash, rebuild_threshold(h));
-  PTS_CHECK_LAUNCH(h);
-  return PTSTORE_OK;
-}
-
-// drop phase: tier, mode EV_DROP (victims -> caller) or EV_HOST_ROOM (victims -> scratch)
-int run_drop(ptstore* h, int tier, int mode, u32 n, int* n_evicted, int* victims, cudaStream_t s) {
-  const int cap = h->sms * 8;
-  const bool two_tier = h->cfg.host_blocks > 0;
-  evict_begin_kernel<<<1, 1, 0, s>>>(h->st, mode, n);
-  PTS_CHECK_LAUNCH(h);
-  unsigned char* blocked = nullptr;
-  if (tier == 1 && two_tier) {
-    blocked = h->blocked;
-    if (cudaMemsetAsync(blocked, 0, (size_t)h->cfg.hbm_blocks + h->cfg.host_blocks, s) != cudaSuccess) {
-      h->last_cuda = (int)cudaGetLastError();
-      return PTSTORE_E_CUDA;
-    }
-    mark_blocked_kernel<<<grid_for(h->cfg.hbm_blocks, 256, cap), 256, 0, s>>>(h->st, blocked);
-    PTS_CHECK_LAUNCH(h);
-  }
-  const u32 span = tier ? h->cfg.host_blocks : h->cfg.hbm_blocks;
-  collect_kernel<<<grid_for(span, 256, cap), 256, 0, s>>>(h->st, tier, blocked, h->sort_buf[0]);
-  PTS_CHECK_LAUNCH(h);
-  int res;
-  int rc = launch_sort(h, s, &res);
-  if (rc) return rc;
-  apply_drop_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, tier, h->sort_buf[res], mode == EV_DROP ? victims : h->room);
-  PTS_CHECK_LAUNCH(h);
-  drop_finish_kernel<<<1, 1, 0, s>>>(h->st, tier, mode, h->sort_buf[res], n_evicted);
-  PTS_CHECK_LAUNCH(h);
-  return PTSTORE_OK;
-}
-
-// make `s` wait for a demotion copy that ptstore_evict_async left running on the side stream
+// make `s` wait for a demotion copy left running on the side stream
 int join_tier(ptstore* h, cudaStream_t s) {
   if (!h->tier_pending) return PTSTORE_OK;
   if (cudaStreamWaitEvent(s, h->ev_copy, 0) != cudaSuccess) { h->last_cuda = (int)cudaGetLastError(); return PTSTORE_E_CUDA; }
@@ -400,28 +334,45 @@ int join_tier(ptstore* h, cudaStream_t s) {
   return PTSTORE_OK;
 }
 
-int evict_impl(ptstore* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, cudaStream_t s, bool async_copy) {
-  if (!h || n_blocks < 0 || (tier != PTSTORE_TIER_HBM && tier != PTSTORE_TIER_HOST) || !n_evicted) return PTSTORE_E_INVAL;
-  if (tier == PTSTORE_TIER_HOST && h->cfg.host_blocks == 0) return PTSTORE_E_INVAL;
+// one phase of an eviction: a single cooperative launch
+int launch_evict(ptstore* h, int tier, int mode, EvictArgs a, cudaStream_t s) {
+  const u32 span = tier ? h->cfg.host_blocks : h->cfg.hbm_blocks;
+  int grid = (int)((span + 511) / 512);
+  if (grid < 1) grid = 1;
+  if (grid > h->coop_grid) grid = h->coop_grid;
+  const u32 per = (span + grid - 1) / grid;
+  a.tier = tier;
+  a.mode = mode;
+  a.tile_elems = (per + EV_THREADS - 1) / EV_THREADS * EV_THREADS;
+  a.room = h->room;
+  a.buf[0] = h->sort_buf[0]; a.buf[1] = h->sort_buf[1];
+  a.hist = h->hist;
+  a.tile_stats = h->tile_stats;
+  a.blocked = (tier == 1 && h->cfg.host_blocks) ? h->blocked : nullptr;
+  a.desc_tier = h->desc_tier;
+  return launch_coop(h, evict_kernel, grid, EV_THREADS, a, s);
+}
+
+// n victims (want_free < 0) or as many as bring the HBM free count to want_free - sum(minus) (decided on the device)
+int evict_impl(ptstore* h, int32_t tier, u32 n, long long want_free, const int* minus, int n_minus, int32_t* n_evicted,
+               int32_t* victim_ids, u32 max_victims, cudaStream_t s, bool async_copy) {
   int rc = join_tier(h, s);
   if (rc) return rc;
-  const u32 n = (u32)n_blocks;
-  if (tier == PTSTORE_TIER_HOST || h->cfg.host_blocks == 0) return run_drop(h, tier, EV_DROP, n, n_evicted, victim_ids, s);
+  EvictArgs a = {};
+  a.n = n; a.want_free = want_free; a.minus = minus; a.n_minus = n_minus; a.max_victims = max_victims;
+  a.n_evicted = n_evicted; a.victims = victim_ids;
+  if (tier == PTSTORE_TIER_HOST || h->cfg.host_blocks == 0) return launch_evict(h, tier, EV_DROP, a, s);
   // HBM tier with a host tier behind it: make room in the host ring, then demote
-  rc = run_drop(h, 1, EV_HOST_ROOM, n, nullptr, nullptr, s);
+  EvictArgs room = a;
+  room.n_evicted = nullptr; room.victims = nullptr;
+  rc = launch_evict(h, 1, EV_HOST_ROOM, room, s);
   if (rc) return rc;
-  const int cap = h->sms * 8;
-  evict_begin_kernel<<<1, 1, 0, s>>>(h->st, EV_DEMOTE, n);
-  PTS_CHECK_LAUNCH(h);
-  collect_kernel<<<grid_for(h->cfg.hbm_blocks, 256, cap), 256, 0, s>>>(h->st, 0, nullptr, h->sort_buf[0]);
-  PTS_CHECK_LAUNCH(h);
-  int res;
-  rc = launch_sort(h, s, &res);
+  if (async_copy) {
+    if (++h->flight_seq == 0) h->flight_seq = 1;
+    a.flight_seq = h->flight_seq;
+  }
+  rc = launch_evict(h, 0, EV_DEMOTE, a, s);
   if (rc) return rc;
-  apply_demote_kernel<<<grid_for(n ? n : 1, 256, cap), 256, 0, s>>>(h->st, h->sort_buf[res], h->desc_tier, victim_ids);
-  PTS_CHECK_LAUNCH(h);
-  demote_finish_kernel<<<1, 256, 0, s>>>(h->st, h->sort_buf[res], n_evicted, victim_ids, h->room);
-  PTS_CHECK_LAUNCH(h);
   Paged none = {};
   if (!async_copy) return launch_copy<COPY_POOL>(h, none, true, s, h->desc_tier, &h->st.ctrl->n_pairs_tier, h->host_ctas);
   // the copy HBM -> host goes to the side stream, ordered after the metadata kernels above
@@ -444,6 +395,60 @@ int evict_impl(ptstore* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, i
   h->tier_pending = true;
   return PTSTORE_OK;
 }
+
+// the linking record of the next fetch call
+int next_fetch_link(ptstore* h, const ptstore_paged_cache_t* dst, const int32_t* block_tables, cudaStream_t s, FetchLink* fl) {
+  if (++h->fetch_seq == 0) {          // the tag wrapped: heads written 2^32 calls ago would look current
+    const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
+    if (cudaMemsetAsync(h->heads, 0, N * 8, s) != cudaSuccess || cudaMemsetAsync(h->st.ctrl->f_pairs, 0, 6 * sizeof(u32), s) != cudaSuccess) {
+      h->last_cuda = (int)cudaGetLastError();
+      return PTSTORE_E_CUDA;
+    }
+    h->fetch_seq = 1;
+  }
+  fl->bt = block_tables;
+  fl->cache_blocks = dst->num_blocks;
+  fl->seq = h->fetch_seq;
+  fl->pending_seq = h->tier_pending ? h->flight_seq : 0;
+  fl->heads = h->heads;
+  fl->node = h->links;
+  fl->desc = h->desc;
+  fl->desc_host = h->desc_host;
+  return PTSTORE_OK;
+}
+
+// the copies of a fetch whose lists have been linked under tag `seq`
+int launch_fetch_copies(ptstore* h, const ptstore_paged_cache_t* dst, u32 seq, cudaStream_t s) {
+  Paged pc = to_paged(dst);
+  pc.head = h->heads;
+  pc.node = h->links;
+  Ctrl* c = h->st.ctrl;
+  const u32 slot = seq & 1u;
+  int rc = launch_copy<COPY_FETCH_MULTI>(h, pc, false, s, h->desc, &c->f_pairs[slot], 0, &c->f_work[slot]);     // HBM-tier sources: every SM
+  if (rc || h->cfg.host_blocks == 0) return rc;
+  return launch_copy<COPY_FETCH_MULTI>(h, pc, true, s, h->desc_host, &c->f_pairs_host[slot], h->host_ctas);       // host-tier sources
+}
+
+int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks, uint32_t flags,
+                int32_t* matched_blocks, int32_t* block_ids, const FetchLink& fl, cudaStream_t s) {
+  const long long* off = reinterpret_cast<const long long*>(offsets);
+  if (split_path(h, R, max_blocks)) {
+    int rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
+    if (rc) return rc;
+    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, fl);
+    PTS_CHECK_LAUNCH(h);
+    return PTSTORE_OK;
+  }
+  switch (lanes_for(h, R, max_blocks)) {
+    case 4: return launch_lookup<4>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, fl, s);
+    case 8: return launch_lookup<8>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, fl, s);
+    case 16: return launch_lookup<16>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, fl, s);
+    default: return launch_lookup<32>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, fl, s);
+  }
+}
+
+template <int L>
+int launch_insert(ptstore* h, InsertArgs& a, int grid, cudaStream_t s) { return launch_coop(h, insert_kernel<L>, grid, INS_THREADS, a, s); }
 
 }  // namespace
 
@@ -468,23 +473,26 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->cfg = *cfg;
   h->lay = lay;
   if (cudaSetDevice(cfg->device) != cudaSuccess) { h->last_cuda = (int)cudaGetLastError(); delete h; return PTSTORE_E_CUDA; }
-  int sms = 0;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0) {
+  int sms = 0, coop = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0 ||
+      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, cfg->device) != cudaSuccess || !coop) {
     (void)cudaGetLastError(); delete h; return PTSTORE_E_CUDA;
   }
   h->sms = sms;
-  h->has_env_tune = env_bulk_tune(&h->env_tune);
+  h->coop_grid = sms < (int)MAX_COOP_GRID ? sms : (int)MAX_COOP_GRID;
+  h->wait_limit = BULK_POLL_LIMIT;
   unsigned char* w = static_cast<unsigned char*>(cfg->workspace);
   h->stash = reinterpret_cast<Slot*>(w + lay.table[1]);
   Store& st = h->st;
   st.table = reinterpret_cast<Slot*>(w + lay.table[0]);
-  st.slots = cfg->table_slots;
+  st.slots = effective_slots(cfg);
   st.m_key = reinterpret_cast<u64*>(w + lay.m_key);
   st.m_parent = reinterpret_cast<u64*>(w + lay.m_parent);
   st.m_last = reinterpret_cast<u64*>(w + lay.m_last);
   st.m_freq = reinterpret_cast<u32*>(w + lay.m_freq);
   st.m_ref = reinterpret_cast<u32*>(w + lay.m_ref);
   st.m_depth = reinterpret_cast<u32*>(w + lay.m_depth);
+  st.m_flight = reinterpret_cast<u32*>(w + lay.m_flight);
   st.ring_ids[0] = reinterpret_cast<int*>(w + lay.ring[0]);
   st.ring_ids[1] = reinterpret_cast<int*>(w + lay.ring[1]);
   st.n[0] = cfg->hbm_blocks; st.n[1] = cfg->host_blocks;
@@ -501,6 +509,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->sort_buf[0] = reinterpret_cast<Key2*>(w + lay.sort[0]);
   h->sort_buf[1] = reinterpret_cast<Key2*>(w + lay.sort[1]);
   h->hist = reinterpret_cast<u32*>(w + lay.hist);
+  h->tile_stats = reinterpret_cast<u64*>(w + lay.tile_stats);
   h->room = reinterpret_cast<int*>(w + lay.room);
   h->desc = reinterpret_cast<int2*>(w + lay.desc);
   h->keys = reinterpret_cast<u64*>(w + lay.keys);
@@ -509,22 +518,18 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->prefix = reinterpret_cast<u32*>(w + lay.prefix);
   h->promo_first = reinterpret_cast<u32*>(w + lay.promo_first);
   h->promo_cnt = reinterpret_cast<u32*>(w + lay.promo_cnt);
+  h->heads = reinterpret_cast<u64*>(w + lay.heads);
   h->links = reinterpret_cast<int2*>(w + lay.links);
   h->desc_tier = reinterpret_cast<int2*>(w + lay.desc_tier);
   h->desc_host = reinterpret_cast<int2*>(w + lay.desc_host);
-  {
-    // a few CTAs saturate the host link; keeping these grids small leaves the SMs to kernels that run beside them
-    const char* e = std::getenv("PTSTORE_HOST_CTAS");
-    const int v = e ? std::atoi(e) : 0;
-    h->host_ctas = v > 0 ? v : 32;
-  }
+  h->host_ctas = 32;     // a few CTAs saturate the host link; a small grid leaves the SMs to kernels that run beside it
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int cap = sms * 8;
   auto fail = [&](int code) { delete h; return code; };
-  table_clear_kernel<<<grid_for((long long)cfg->table_slots, 256, cap), 256, 0, s>>>(st.table, cfg->table_slots);
+  table_clear_kernel<<<grid_for((long long)st.slots, 256, cap), 256, 0, s>>>(st.table, st.slots);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
-  store_init_kernel<<<grid_for((long long)cfg->hbm_blocks + cfg->host_blocks, 256, cap), 256, 0, s>>>(st);
+  store_init_kernel<<<grid_for((long long)cfg->hbm_blocks + cfg->host_blocks, 256, cap), 256, 0, s>>>(st, h->heads);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
   ctrl_init_kernel<<<1, 1, 0, s>>>(st);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
@@ -570,21 +575,29 @@ int ptstore_lookup(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   if (R > 0 && (!offsets || !matched_blocks || !block_ids)) return PTSTORE_E_INVAL;
   h->epoch += 1;
   if (R == 0) return PTSTORE_OK;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const long long* off = reinterpret_cast<const long long*>(offsets);
-  if (split_path(h, R, max_blocks)) {
-    rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
+  FetchLink none = {};
+  return lookup_impl(h, tokens, offsets, R, max_blocks, flags, matched_blocks, block_ids, none, static_cast<cudaStream_t>(stream));
+}
+
+int ptstore_lookup_fetch(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks, uint32_t flags,
+                         const ptstore_paged_cache_t* dst, const int32_t* block_tables, int32_t* matched_blocks, int32_t* block_ids,
+                         ptstore_stream_t stream) {
+  int rc = check_batch(h, R, max_blocks);
+  if (rc) return rc;
+  if (R > 0 && (!offsets || !matched_blocks || !block_ids || !block_tables)) return PTSTORE_E_INVAL;
+  if (R > 0) {
+    rc = check_cache(h, dst);
     if (rc) return rc;
-    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids);
-    PTS_CHECK_LAUNCH(h);
-    return PTSTORE_OK;
   }
-  switch (lanes_for(h, R, max_blocks)) {
-    case 4: return launch_lookup<4>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
-    case 8: return launch_lookup<8>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
-    case 16: return launch_lookup<16>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
-    default: return launch_lookup<32>(h, tokens, off, R, max_blocks, flags, matched_blocks, block_ids, s);
-  }
+  h->epoch += 1;
+  if (R == 0) return PTSTORE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  FetchLink fl;
+  rc = next_fetch_link(h, dst, block_tables, s, &fl);
+  if (rc) return rc;
+  rc = lookup_impl(h, tokens, offsets, R, max_blocks, flags, matched_blocks, block_ids, fl, s);
+  if (rc) return rc;
+  return launch_fetch_copies(h, dst, fl.seq, s);
 }
 
 int ptstore_fetch(ptstore_t* h, const int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
@@ -596,20 +609,13 @@ int ptstore_fetch(ptstore_t* h, const int32_t* block_ids, const int32_t* matched
   rc = check_cache(h, dst);
   if (rc) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // one descriptor per distinct source block, each with the list of its destinations (promo_first doubles as the list heads)
-  const u32 n_blocks = h->cfg.hbm_blocks + h->cfg.host_blocks;
-  const int cap = h->sms * 8;
-  fetch_begin_kernel<<<grid_for(n_blocks, 256, cap), 256, 0, s>>>(h->st, h->promo_first, n_blocks);
+  // one descriptor per distinct source block, each with the list of its destinations
+  FetchLink fl;
+  rc = next_fetch_link(h, dst, block_tables, s, &fl);
+  if (rc) return rc;
+  fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, block_ids, matched_blocks, R, max_blocks, fl);
   PTS_CHECK_LAUNCH(h);
-  fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, block_tables, R, max_blocks,
-                                                                                 dst->num_blocks, h->promo_first, h->links, h->desc, h->desc_host);
-  PTS_CHECK_LAUNCH(h);
-  Paged pc = to_paged(dst);
-  pc.head = h->promo_first;
-  pc.node = h->links;
-  rc = launch_copy<COPY_FETCH_MULTI>(h, pc, false, s);                    // HBM-tier sources: every SM
-  if (rc || h->cfg.host_blocks == 0) return rc;
-  return launch_copy<COPY_FETCH_MULTI>(h, pc, true, s, h->desc_host, &h->st.ctrl->n_pairs_host, h->host_ctas);   // host-tier sources
+  return launch_fetch_copies(h, dst, fl.seq, s);
 }
 
 int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
@@ -629,33 +635,34 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   rc = join_tier(h, s);        // new blocks may reuse HBM ids whose demotion copy is still running
   if (rc) return rc;
-  rc = maybe_rebuild(h, s);
-  if (rc) return rc;
-  const long long* off = reinterpret_cast<const long long*>(offsets);
-  if (split_path(h, R, max_blocks)) rc = launch_hash_split(h, tokens, off, R, max_blocks, h->keys, s);
-  else switch (lanes_for(h, R, max_blocks)) {
-    case 4: rc = launch_hash<4>(h, tokens, off, R, max_blocks, h->keys, s); break;
-    case 8: rc = launch_hash<8>(h, tokens, off, R, max_blocks, h->keys, s); break;
-    case 16: rc = launch_hash<16>(h, tokens, off, R, max_blocks, h->keys, s); break;
-    default: rc = launch_hash<32>(h, tokens, off, R, max_blocks, h->keys, s); break;
+  const long long total = (long long)R * max_blocks;
+  InsertArgs a = {};
+  a.tokens = tokens;
+  a.offsets = reinterpret_cast<const long long*>(offsets);
+  a.R = R; a.max_blocks = max_blocks;
+  a.split = split_path(h, R, max_blocks) ? 1 : 0;
+  a.keys = h->keys; a.eslot = h->eslot; a.cta_sums = h->cta_sums;
+  a.bt = copy ? block_tables : nullptr;
+  a.cache_blocks = copy ? src->num_blocks : 0;
+  a.epoch = h->epoch;
+  a.desc = h->desc;
+  a.ids_out = block_ids; a.new_blocks = new_blocks;
+  a.stash = h->stash;
+  a.rebuild_threshold = rebuild_threshold(h);
+  const int lanes = a.split ? 32 : lanes_for(h, R, max_blocks);
+  // CTAs: enough for one element per thread and for one sub-warp per request, at most one per SM
+  const long long by_elems = (total + INS_THREADS - 1) / INS_THREADS;
+  const long long by_reqs = ((long long)R * lanes + INS_THREADS - 1) / INS_THREADS;
+  long long g = by_elems > by_reqs ? by_elems : by_reqs;
+  const int grid = (int)(g < 1 ? 1 : (g > h->coop_grid ? h->coop_grid : g));
+  switch (lanes) {
+    case 4: rc = launch_insert<4>(h, a, grid, s); break;
+    case 8: rc = launch_insert<8>(h, a, grid, s); break;
+    case 16: rc = launch_insert<16>(h, a, grid, s); break;
+    default: rc = launch_insert<32>(h, a, grid, s); break;
   }
   if (rc) return rc;
-  const long long total = (long long)R * max_blocks;
-  const int cap = h->sms * 8;
-  insert_claim_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, h->keys, R, max_blocks, h->eslot, new_blocks);
-  PTS_CHECK_LAUNCH(h);
-  const u32 n_ctas = (u32)((total + INS_THREADS - 1) / INS_THREADS);
-  insert_count_kernel<<<n_ctas, INS_THREADS, 0, s>>>(h->st, h->eslot, total, max_blocks, h->cta_sums);
-  PTS_CHECK_LAUNCH(h);
-  insert_plan_kernel<<<1, INS_THREADS, 0, s>>>(h->st, h->cta_sums, n_ctas, rebuild_threshold(h));
-  PTS_CHECK_LAUNCH(h);
-  insert_assign_kernel<<<n_ctas, INS_THREADS, 0, s>>>(h->st, h->keys, h->eslot, total, max_blocks, h->cta_sums,
-                                                       copy ? block_tables : nullptr, copy ? src->num_blocks : 0, h->epoch, h->desc,
-                                                       new_blocks);
-  PTS_CHECK_LAUNCH(h);
-  insert_finish_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, h->eslot, total, h->epoch, block_ids);
-  PTS_CHECK_LAUNCH(h);
-  if (copy) return launch_copy<COPY_INSERT>(h, to_paged(src), false, s);
+  if (copy) return launch_copy<COPY_INSERT>(h, to_paged(src), false, s, h->desc, &h->st.ctrl->n_pairs);
   return PTSTORE_OK;
 }
 
@@ -671,12 +678,27 @@ int ptstore_release(ptstore_t* h, const int32_t* block_ids, const int32_t* match
   return PTSTORE_OK;
 }
 
+static int evict_entry(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, ptstore_stream_t stream, bool async_copy) {
+  if (!h || n_blocks < 0 || (tier != PTSTORE_TIER_HBM && tier != PTSTORE_TIER_HOST) || !n_evicted) return PTSTORE_E_INVAL;
+  if (tier == PTSTORE_TIER_HOST && h->cfg.host_blocks == 0) return PTSTORE_E_INVAL;
+  return evict_impl(h, tier, (u32)n_blocks, -1, nullptr, 0, n_evicted, victim_ids, 0xFFFFFFFFu, static_cast<cudaStream_t>(stream), async_copy);
+}
+
 int ptstore_evict(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, ptstore_stream_t stream) {
-  return evict_impl(h, tier, n_blocks, n_evicted, victim_ids, static_cast<cudaStream_t>(stream), false);
+  return evict_entry(h, tier, n_blocks, n_evicted, victim_ids, stream, false);
 }
 
 int ptstore_evict_async(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n_evicted, int32_t* victim_ids, ptstore_stream_t stream) {
-  return evict_impl(h, tier, n_blocks, n_evicted, victim_ids, static_cast<cudaStream_t>(stream), true);
+  return evict_entry(h, tier, n_blocks, n_evicted, victim_ids, stream, true);
+}
+
+int ptstore_reserve(ptstore_t* h, int64_t want_free, const int32_t* minus, int32_t n_minus, uint32_t flags, int32_t* n_evicted,
+                    int32_t* victim_ids, int32_t max_victims, ptstore_stream_t stream) {
+  if (!h || want_free < 0 || n_minus < 0 || (n_minus > 0 && !minus) || !n_evicted || max_victims < 0) return PTSTORE_E_INVAL;
+  if ((u32)n_minus > h->cfg.max_requests) return PTSTORE_E_LIMIT;
+  const u32 cap = victim_ids ? (u32)max_victims : 0x7FFFFFFFu;
+  return evict_impl(h, PTSTORE_TIER_HBM, 0, (long long)want_free, minus, n_minus, n_evicted, victim_ids, cap,
+                    static_cast<cudaStream_t>(stream), (flags & PTSTORE_ASYNC_COPY) != 0);
 }
 
 int ptstore_join(ptstore_t* h, ptstore_stream_t stream) {
@@ -718,7 +740,20 @@ int ptstore_promote(ptstore_t* h, int32_t* block_ids, const int32_t* matched_blo
   promote_rewrite_kernel<<<grid_for(total, 256, cap), 256, 0, s>>>(h->st, block_ids, matched_blocks, total, max_blocks, h->promo_first);
   PTS_CHECK_LAUNCH(h);
   Paged none = {};
-  return launch_copy<COPY_POOL>(h, none, true, s, nullptr, nullptr, h->host_ctas);      // host -> HBM at host-link speed
+  return launch_copy<COPY_POOL>(h, none, true, s, h->desc, &h->st.ctrl->n_pairs, h->host_ctas);      // host -> HBM at host-link speed
+}
+
+int ptstore_time_next_copy(ptstore_t* h, void* before, void* after) {
+  if (!h || !before || !after) return PTSTORE_E_INVAL;
+  h->time_before = static_cast<cudaEvent_t>(before);
+  h->time_after = static_cast<cudaEvent_t>(after);
+  return PTSTORE_OK;
+}
+
+int ptstore_set_wait_limit(ptstore_t* h, uint32_t polls) {
+  if (!h) return PTSTORE_E_INVAL;
+  h->wait_limit = polls ? polls : BULK_POLL_LIMIT;
+  return PTSTORE_OK;
 }
 
 int ptstore_status(ptstore_t* h, ptstore_stream_t stream, uint32_t* status_out) {

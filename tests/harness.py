@@ -54,6 +54,32 @@ class Pair:
         assert (io == ig.cpu().numpy()).all(), "block ids differ"
         return mo, io, mg, ig
 
+    def lookup_fetch(self, seqs, max_blocks, np_cache, block_tables, flags=0):
+        """The fused call against the oracle's lookup followed by its fetch (np_cache is modified by the oracle)."""
+        toks, offs = W.ragged(seqs)
+        gc = self.gpu_cache(np_cache)
+        mo, io = self.o.lookup(toks, offs, max_blocks, flags)
+        self.o.fetch(io, mo, np_cache, block_tables)
+        mg, ig = self.g.lookup_fetch(dev(toks), dev(offs), max_blocks, gc, dev(block_tables), flags)
+        assert (mo == mg.cpu().numpy()).all(), "matched lengths differ"
+        assert (io == ig.cpu().numpy()).all(), "block ids differ"
+        for l in range(self.shape.layers):
+            assert torch.equal(gc.tensors[l].cpu(), torch.from_numpy(np_cache[l])), "fetched bytes differ in layer %d" % l
+        return mo, io
+
+    def reserve(self, want_free, minus, literal=True, asynchronous=False, max_victims=None):
+        """ptstore_reserve against the oracle's evict of the count the definition gives."""
+        n = max(0, int(want_free) - int(np.maximum(minus, 0).sum()) - self.o.free_count(0))
+        cap = n if max_victims is None else max_victims
+        n = min(n, cap)
+        ne_o, v_o = self.o.evict(0, n, literal=literal)
+        ne_g, v_g = self.g.reserve(want_free, dev(minus.astype(np.int32)), G.ASYNC_COPY if asynchronous else 0, max_victims=max(cap, 1))
+        ne_g = ne_g.cpu().numpy()
+        assert ne_o.tolist() == ne_g.tolist(), ("evicted counts differ", ne_o, ne_g)
+        k = int(ne_o.sum())
+        assert v_o.tolist() == v_g.cpu().numpy()[:k].tolist(), "victims differ"
+        return ne_o, v_o
+
     def fetch(self, ids, matched, np_cache, block_tables):
         """np_cache is modified by the oracle; a device copy of its ORIGINAL content by the library; then compared."""
         gc = self.gpu_cache(np_cache)

@@ -25,7 +25,7 @@ def test_header_symbols_are_exported():
 def test_binding_declares_the_same_entry_points():
     src = open(os.path.join(ROOT, "paper_2607_22648_b200", "binding.py")).read()
     listed = set(re.findall(r'"(ptstore_[a-z_]+)"', src))
-    assert set(declared_functions()) <= listed | {"ptstore_evict_static"} or set(declared_functions()) <= listed
+    assert set(declared_functions()) <= listed
 
 
 def test_host_only_calls_validate_arguments():

@@ -36,7 +36,8 @@ def test_llama8b_pool20k_batch64_serving_steps(policy):
     srv = LockstepServing(sh, pool, 0, 64, mb, cache_blocks, seed=2, policy=policy)
     seen_evict = False
     for k, (seqs, tags) in enumerate(batches):
-        r = srv.step(seqs, tags, sample=80, check_all=True, poison=(k == 3))
+        # even steps: the fused calls the benchmark times; odd steps: the separate calls
+        r = srv.step(seqs, tags, sample=80, check_all=True, poison=(k == 3), fused=(k % 2 == 0))
         seen_evict |= r["evicted"] is not None
         assert r["status"] == 0
     s = srv.check_counts()
@@ -91,7 +92,7 @@ def test_llama70b_16k_prefix_fetch_shuffled_tables():
     srv = LockstepServing(sh, pool, 0, 8, mb, cache_blocks, seed=4)
     for k in range(4):
         seqs, tags = st.batch(8)
-        r = srv.step(seqs, tags, sample=100, check_all=(k >= 2), poison=(k == 3))
+        r = srv.step(seqs, tags, sample=100, check_all=(k >= 2), poison=(k == 3), fused=(k == 2))
     assert r["matched"] >= 4 * 512                          # Zipf(1.2) over 18 documents: most of the batch hits
     srv.check_counts()
     assert srv.check_pool(8) > 0
@@ -116,7 +117,8 @@ def test_churn_with_host_tier():
     demoted = dropped = promoted = 0
     for k in range(n_steps):
         seqs, tags = st.batch(16)
-        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9), promote=(256 if k >= 30 else 0), async_demote=(k >= 20 and k % 2 == 0))
+        r = srv.step(seqs, tags, sample=6, check_all=(k % 10 == 9), promote=(256 if k >= 30 else 0), async_demote=(k >= 20 and k % 2 == 0),
+                     fused=(k < 20 and k % 4 == 3))
         promoted += r["promoted"]
         if r["evicted"] is not None:
             demoted += int(r["evicted"][0]); dropped += int(r["evicted"][1])
@@ -141,7 +143,7 @@ def test_multi_turn_conversations_grow_chains_by_small_increments():
     hits = evicts = 0
     for k in range(40):
         seqs, tags = st.batch(32)
-        r = srv.step(seqs, tags, sample=8, check_all=(k % 8 == 7))
+        r = srv.step(seqs, tags, sample=8, check_all=(k % 8 == 7), fused=(k % 2 == 1))
         hits += r["matched"]
         evicts += r["evicted"] is not None
         assert r["status"] == 0

@@ -25,10 +25,10 @@ ENGINES = [
     ("bulk_auto", lambda G: G.COPY_BULK),
     ("bulk_8x8k_3cta", lambda G: G.COPY_BULK | G.copy_variant(1)),
     ("bulk_3x32k", lambda G: G.COPY_BULK | G.copy_variant(2)),
-    ("bulk_12x16k", lambda G: G.COPY_BULK | G.copy_variant(5)),
-    ("bulk_group2", lambda G: G.COPY_BULK | G.copy_variant(8)),
-    ("bulk_l2hint", lambda G: G.COPY_BULK | G.copy_variant(9)),
-    ("bulk_3x64k", lambda G: G.COPY_BULK | G.copy_variant(10)),
+    ("bulk_12x16k", lambda G: G.COPY_BULK | G.copy_variant(4)),
+    ("bulk_group2", lambda G: G.COPY_BULK | G.copy_variant(5)),
+    ("bulk_l2hint", lambda G: G.COPY_BULK | G.copy_variant(6)),
+    ("bulk_3x64k", lambda G: G.COPY_BULK | G.copy_variant(7)),
 ]
 
 
@@ -621,3 +621,163 @@ def test_chunk_sizes_that_do_not_divide_into_stages(engine):
         p.fetch(io, mo, dst, bt)
         assert p.check_status() == 0
         p.close()
+
+
+# ---- fused entry points ----------------------------------------------------------------------------------------------
+def _tables_for(rng, matched_upper, n_req, mb, nd):
+    """Block tables with a distinct destination for every (request, block) position that could match."""
+    bt = np.full((n_req, mb), -1, dtype=np.int32)
+    perm, k = rng.permutation(nd), 0
+    for r in range(n_req):
+        for j in range(matched_upper[r]):
+            bt[r, j] = perm[k]
+            k += 1
+    return bt
+
+
+@pytest.mark.parametrize("name,mk", [ENGINES[0], ENGINES[3], ENGINES[4]], ids=["vector", "bulk", "bulk_8x8k_3cta"])
+def test_lookup_fetch_equals_lookup_then_fetch(name, mk):
+    """The fused call on the tiny config: many requests of one block column (sub-warps of 8 and 16 lanes), few long
+    requests (the split path), shared prefixes (several destinations per source block) and misses."""
+    Pair, dev, G = _imports()
+    w = W.tiny()
+    sh, B = w.shape, w.shape.block_tokens
+    rng = np.random.default_rng(5)
+    p = Pair(sh, w.pool_blocks, flags=mk(G), max_requests=1200, max_batch_blocks=1200 * 8)
+    smb = W.max_blocks_of(w.store_seqs, B)
+    for i in range(0, len(w.store_seqs), 16):
+        part = w.store_seqs[i:i + 16]
+        need = sum(len(s) // B for s in part)
+        p.insert(part, smb, W.random_kv_cache(i, sh, need + 3), W.shuffled_block_tables(rng, part, B, smb, need + 3))
+    batches = [
+        (w.queries, W.max_blocks_of(w.queries, B)),                                   # 8 long requests: split path
+        ([w.store_seqs[i % 64] for i in range(40)] + w.queries[:3], 32),              # 43 requests, shared prefixes, L = 32
+        ([w.store_seqs[i % 64][: 8 * B] for i in range(1100)], 8),                    # 1100 short requests: L = 8
+        ([w.store_seqs[i % 64][: 12 * B] for i in range(1030)], 9),                   # capped at 9 blocks, L = 16
+    ]
+    for seqs, mb in batches:
+        upper = [min(len(s) // B, mb) for s in seqs]
+        nd = sum(upper) + 5
+        bt = _tables_for(rng, upper, len(seqs), mb, nd)
+        dst = [np.full((2, nd, sh.chunk_bytes), 0x3C, dtype=np.uint8) for _ in range(sh.layers)]
+        mo, io = p.lookup_fetch(seqs, mb, dst, bt, flags=1)
+        assert mo.sum() > 0
+        if seqs is w.queries:
+            first_matched = mo
+        p.release(io, mo)
+        assert p.check_status() == 0
+    s = p.check_counts()
+    assert s.blocks_fetched[0] == s.blocks_matched
+    # an out-of-range table entry is skipped and flagged exactly as by the separate calls
+    seqs, mb = batches[0]
+    upper = [min(len(x) // B, mb) for x in seqs]
+    nd = sum(upper) + 5
+    bt = _tables_for(rng, upper, len(seqs), mb, nd)
+    r0 = int(np.argmax(first_matched > 0))
+    bt[r0, 0] = nd + 7
+    dst = [np.full((2, nd, sh.chunk_bytes), 0x3C, dtype=np.uint8) for _ in range(sh.layers)]
+    p.lookup_fetch(seqs, mb, dst, bt)
+    assert p.check_status() == G.S_BOUNDS
+    p.close()
+
+
+@pytest.mark.parametrize("host,policy", [(0, "lru"), (20, "lru"), (20, "gdsf")])
+def test_fused_step_lockstep(host, policy):
+    """A serving loop made of the fused calls only: lookup_fetch(PIN) -> reserve -> insert -> release, random batches,
+    compared call by call; with a host tier the reserve demotes (synchronously or with the copy on the side stream)."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(2, 1, 8, 2)
+    B = 2
+    for seed in range(4):
+        rng = np.random.default_rng(700 + seed)
+        p = Pair(sh, 36, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * 12, table_slots=307, policy=policy)
+        seqs = []
+        for step in range(50):
+            base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.75 else np.zeros(0, dtype=np.int32)
+            cut = int(rng.integers(0, len(base) + 1))
+            s = np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(1, 10)), dtype=np.int32)])[:24]
+            seqs.append(s)
+            batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(int(rng.integers(1, 6)))] + [s]
+            mb = 12
+            upper = [len(x) // B for x in batch]
+            nd = sum(upper) + 2
+            bt = _tables_for(rng, upper, len(batch), mb, nd)
+            dst = W.random_kv_cache(seed * 1000 + step, sh, nd)          # holds the new blocks' K/V; hits overwrite their part
+            mo, io = p.lookup_fetch(batch, mb, dst, bt, flags=1)
+            asyn = bool(host) and step % 3 == 0
+            p.reserve(sum(upper), mo, literal=bool(step % 2), asynchronous=asyn, max_victims=40 if step % 5 else 3)
+            p.insert(batch, mb, dst, bt)
+            p.release(io, mo)
+            p.check_status()
+            if step % 10 == 9:
+                p.check_pools()
+                p.check_counts()
+        p.check_pools()
+        p.check_counts()
+        p.close()
+
+
+def test_fetch_of_a_block_in_flight_is_skipped_and_flagged():
+    """After an asynchronous demotion and before the join, a fetch that names a block whose copy may still be running
+    must not read it: the entry is skipped and S_INFLIGHT raised; after the join the same fetch is byte-exact."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(2, 1, 8, 2)
+    p = Pair(sh, 6, host_blocks=6, max_requests=2, max_batch_blocks=8)
+    rng = np.random.default_rng(1)
+    a = np.array([1, 1, 2, 2, 3, 3, 4, 4], dtype=np.int32)
+    src = W.random_kv_cache(1, sh, 4)
+    p.insert([a], 4, src, np.array([[0, 1, 2, 3]], dtype=np.int32))
+    p.evict(0, 2, asynchronous=True)                     # blocks 3 and 2 move to the host tier, copy on the side stream
+    mo, io, mg, ig = p.lookup([a], 4)
+    assert io.tolist() == [[0, 1, 7, 6]]
+    bt = np.array([[0, 1, 2, 3]], dtype=np.int32)
+    cache = p.gpu_cache([np.full((2, 4, sh.chunk_bytes), 0x44, dtype=np.uint8) for _ in range(sh.layers)])
+    p.g.fetch(ig, mg, cache, dev(bt))
+    assert p.g.status() == G.S_INFLIGHT
+    for l in range(sh.layers):
+        got = cache.tensors[l].cpu().numpy()
+        assert (got[:, 2:] == 0x44).all() and (got[:, 0] == src[l][:, 0]).all() and (got[:, 1] == src[l][:, 1]).all()
+    p.g.join()
+    dst = [np.full((2, 4, sh.chunk_bytes), 0x44, dtype=np.uint8) for _ in range(sh.layers)]
+    p.fetch(io, mo, dst, bt)
+    assert p.check_status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("engine", ["bulk", "bulk_multi"])
+def test_bounded_wait_runs_out_and_the_store_stays_usable(engine):
+    """With one poll per wait every copy CTA gives up at its first wait: the call returns, S_TIMEOUT is raised, nothing
+    hangs; with the limit restored the same copy is byte-exact (the CTAs drained what they had in flight)."""
+    Pair, dev, G = _imports()
+    sh = W.LLAMA3_8B
+    B = sh.block_tokens
+    rng = np.random.default_rng(2)
+    p = Pair(sh, 48, max_requests=4, max_batch_blocks=4 * 16)
+    doc = rng.integers(0, 1000, size=12 * B, dtype=np.int32)
+    src = W.random_kv_cache(9, sh, 12)
+    tab = np.arange(12, dtype=np.int32)[None, :].repeat(1, 0)
+    tab16 = np.full((1, 16), -1, dtype=np.int32); tab16[0, :12] = tab[0]
+    if engine == "bulk":                                  # the insert copy uses copy_bulk_kernel
+        p.g.set_wait_limit(1)
+        toks, offs = W.ragged([doc])
+        p.o.insert(toks, offs, 16, src, tab16)
+        p.g.insert(dev(toks), dev(offs), 16, p.gpu_cache(src), dev(tab16))
+        assert p.g.status() & G.S_TIMEOUT
+        p.g.set_wait_limit(0)
+        p.evict(0, 12)                                    # both sides drop the (incompletely copied) blocks
+        p.insert([doc], 16, src, tab16)
+        p.check_pools()
+    else:                                                 # the fetch copy uses copy_bulk_multi_kernel
+        p.insert([doc], 16, src, tab16)
+        mo, io, mg, ig = p.lookup([doc, doc], 16)
+        bt = np.full((2, 16), -1, dtype=np.int32); bt[0, :12] = np.arange(12); bt[1, :12] = np.arange(12, 24)
+        cache = G.PagedKV(sh.layers, 24, sh.chunk_bytes)
+        p.g.set_wait_limit(1)
+        p.g.fetch(ig, mg, cache, dev(bt))
+        assert p.g.status() & G.S_TIMEOUT
+        p.g.set_wait_limit(0)
+        dst = [np.zeros((2, 24, sh.chunk_bytes), dtype=np.uint8) for _ in range(sh.layers)]
+        p.fetch(io, mo, dst, bt)
+    assert p.check_status() == 0
+    p.check_counts()
+    p.close()
