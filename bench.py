@@ -1,19 +1,23 @@
 """Benchmark of the prefix-hit path on B200.
 
 A step is one pass of the whole path over one batch of synthetic prompts:
-    lookup(PIN) -> fetch -> evict(what the batch will need) -> insert -> release
+    lookup_fetch(PIN) -> reserve(room for the batch's new blocks) -> insert -> release
 on the Llama-3-8B KV shape (32 layers x 8 KV heads x 128, bf16, 16-token blocks), a 20,000-block store
 pool in HBM, 500 documents of 2k-6k tokens with Zipf(1.1) popularity, 64 prompts per batch, each a
-document plus a unique 64-256-token question.
+document plus a unique 64-256-token question.  No call waits for the host: matched lengths, free counts and
+the number of victims stay on the device.
 
-Prints ONE JSON line.  `value` is KV bytes moved by fetch and insert (read + write) divided by the
-time of the whole steps, inputs resident in HBM.  `e2e` repeats the measurement with the step's token
-ids / offsets / block tables copied from pinned host memory and its results copied back inside the
-timed region.  `roofline` is the fetch copy kernel alone against the measured HBM copy bandwidth.
-`cpu_baseline` is the CPU oracle timed on this machine on a bounded sample of the same stream.
+Prints ONE JSON line.  `value` is the KV bytes DRAM has to move for the fetches and inserts of the timed steps
+(each distinct source block read once, every delivered or stored block written once, stored blocks read once)
+divided by the time of the whole steps, inputs resident in HBM; `value_delivered_bytes` counts 2 x block bytes
+per delivered block instead.  `e2e` repeats the measurement with the step's token ids / offsets / block tables
+copied from pinned host memory and its results copied back inside the timed region.  `roofline` is the fetch
+copy kernel alone (events recorded around that kernel by the library) against the measured HBM copy bandwidth.
+`latency` holds small-batch steps (1 / 4 / 16 prompts of 4k tokens that hit), `lookup` the 10^6-node lookup
+stress, `cpu_baseline` the CPU oracle timed on this machine on a bounded sample of the same stream.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--engine vector|bulk] ...
-Under torchrun (N > 1) every rank runs an independent replica on its own GPU (the path has no
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload ...] ...
+With --gpus N > 1 (or under torchrun) every rank runs an independent replica on its own GPU (the path has no
 exchange step); rank 0 prints the aggregate.
 """
 import argparse
@@ -34,10 +38,12 @@ from paper_2607_22648_b200 import workloads as W  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes of the fetch copy kernel per block, from the ncu capture of a small case (profiles/): traffic grows in
-# proportion to the blocks read and written, so a full launch is these factors times its block counts.
+# proportion to the blocks read and written, so a full launch is MODELLED as these factors times its block counts.
 NCU_READ_FACTOR = 1.00    # dram__bytes_read.sum / (distinct source blocks x block bytes)
 NCU_WRITE_FACTOR = 0.99   # dram__bytes_write.sum / (delivered blocks x block bytes)
 FALLBACK_HBM_GBS = 6650.0
+# L2 read sectors per issued probe of lookup_kernel on the 10^6-node stress, from the ncu capture in profiles/
+L2_SECTORS_PER_PROBE = 9.4
 
 
 def measured_peak():
@@ -193,60 +199,65 @@ class Serving:
         self.h_matched = torch.empty(R, dtype=torch.int32).pin_memory()
         self.h_ids = torch.empty((R, self.mb), dtype=torch.int32).pin_memory()
         self.h_newb = torch.empty(R, dtype=torch.int32).pin_memory()
-        self.h_stats = torch.zeros(ctypes_sizeof_stats(self.G), dtype=torch.uint8).pin_memory()
-        self.after_lookup = torch.cuda.Event()
 
     def step(self, i, e2e=False, events=None):
-        """One pass of the path.  Returns nothing; counters come from ptstore_stats."""
+        """One pass of the path.  Returns nothing; counters come from ptstore_stats.  No host synchronisation inside."""
         torch, G, st = self.torch, self.G, self.store
         s = self.steps[i]
         if e2e:
             d = {k: v.to("cuda", non_blocking=True) for k, v in s["host"].items()}
         else:
             d = s["dev"]
-        st.lookup(d["tokens"], d["offsets"], self.mb, G.PIN, self.matched, self.ids)
-        if self.promote:
-            if events is not None:
-                events["promote"].append((self._ev(), None))
-            st.promote(self.ids, self.matched, G.PINNED_LIST, self.promote, self.nprom)
-            if events is not None:
-                events["promote"][-1] = (events["promote"][-1][0], self._ev())
-        self.h_matched.copy_(self.matched, non_blocking=True)
-        st.stats_enqueue(self.h_stats)
-        self.after_lookup.record()
-        if self.async_demote:
-            self._evict_shortfall(s, events)          # its demotion copy (device -> host) overlaps the fetch (host -> device)
-        if events is not None:
-            events["fetch"].append((self._ev(), None))
-        st.fetch(self.ids, self.matched, self.cache, d["bt"])
-        if events is not None:
-            events["fetch"][-1] = (events["fetch"][-1][0], self._ev())
-        if not self.async_demote:
-            self._evict_shortfall(s, events)
-        if events is not None:
-            events["insert"].append((self._ev(), None))
+        want = s["total_blocks"] + self.promote              # free HBM blocks the insert needs (+ room for the next promotions)
+        timed = events is not None
+        if self.promote or self.async_demote:                # promotion sits between lookup and fetch; an asynchronous
+            st.lookup(d["tokens"], d["offsets"], self.mb, G.PIN, self.matched, self.ids)     # demotion starts before the fetch
+            if self.promote:
+                a = self._ev() if timed else None
+                st.promote(self.ids, self.matched, G.PINNED_LIST, self.promote, self.nprom)
+                if timed:
+                    events["promote"].append((a, self._ev()))
+            if self.async_demote:
+                self._reserve(want, G.ASYNC_COPY, events)    # its copy (device -> host) overlaps the fetch (host -> device)
+            a = self._ev() if timed else None
+            if timed:
+                self._time_copy(events["fetch_copy"])
+            st.fetch(self.ids, self.matched, self.cache, d["bt"])
+            if timed:
+                events["fetch"].append((a, self._ev()))
+            if not self.async_demote:
+                self._reserve(want, 0, events)
+        else:
+            a = self._ev() if timed else None
+            if timed:
+                self._time_copy(events["fetch_copy"])
+            st.lookup_fetch(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], G.PIN, self.matched, self.ids)
+            if timed:
+                events["fetch"].append((a, self._ev()))
+            self._reserve(want, 0, events)
+        a = self._ev() if timed else None
+        if timed:
+            self._time_copy(events["insert_copy"])
         st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb)
-        if events is not None:
-            events["insert"][-1] = (events["insert"][-1][0], self._ev())
+        if timed:
+            events["insert"].append((a, self._ev()))
         st.release(self.ids, self.matched)
         if e2e:
+            self.h_matched.copy_(self.matched, non_blocking=True)
             self.h_ids.copy_(self.ids, non_blocking=True)
             self.h_newb.copy_(self.newb, non_blocking=True)
 
-    def _evict_shortfall(self, s, events):
-        # the serving engine needs the matched lengths on the host anyway; the counters come back with them, behind an event
-        # recorded right after the lookup, so the host does not wait for the fetch that is already queued
-        torch, G, st = self.torch, self.G, self.store
-        self.after_lookup.synchronize()
-        stats = G.Stats.from_buffer_copy(self.h_stats.numpy().tobytes())
-        need = s["total_blocks"] - int(self.h_matched.sum()) + self.promote      # keep room for the next step's promotions
-        short = need - int(stats.free_blocks[0])
-        if short > 0:
-            if events is not None:
-                events["evict"].append((self._ev(), None))
-            st.evict(G.TIER_HBM, short, want_victims=False, n_evicted=self.nev, asynchronous=self.async_demote)
-            if events is not None:
-                events["evict"][-1] = (events["evict"][-1][0], self._ev())
+    def _reserve(self, want, flags, events):
+        a = self._ev() if events is not None else None
+        self.store.reserve(want, self.matched, flags, n_evicted=self.nev)
+        if events is not None:
+            events["evict"].append((a, self._ev()))
+
+    def _time_copy(self, sink):
+        """Have the library record two events around the next HBM copy kernel."""
+        a, b = self._ev(), self._ev()
+        self.store.time_next_copy(a, b)
+        sink.append((a, b))
 
     def _ev(self):
         e = self.torch.cuda.Event(enable_timing=True)
@@ -258,11 +269,6 @@ class Serving:
         h2d = sum(v.numel() * v.element_size() for v in s["host"].values())
         d2h = self.h_matched.numel() * 4 + self.h_ids.numel() * 4 + self.h_newb.numel() * 4
         return h2d, d2h
-
-
-def ctypes_sizeof_stats(G):
-    import ctypes
-    return ctypes.sizeof(G.Stats)
 
 
 def reduce_over_ranks(dist, x, op, device):
@@ -282,17 +288,60 @@ def whole_job_throughput(dist, ms, nbytes, device):
     return ms_all, bytes_all, bytes_all / (ms_all * 1e-3) / 1e9
 
 
-def run_gpu(args):
-    import torch
+def init_ranks(backend):
+    """(rank, world, local rank, dist or None) from the launcher's environment; one process per GPU."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     dist = None
     if world > 1:
+        import torch
         import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
+        if backend == "nccl":
+            if local >= torch.cuda.device_count():
+                raise SystemExit("rank %d has no GPU: %d ranks on %d visible devices" % (rank, world, torch.cuda.device_count()))
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group("gloo")
+    return rank, world, local, dist
+
+
+def relaunch_as_replicas(args):
+    """`--gpus N` outside a launcher: start N ranks of this script, one per GPU, and let them report."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=%d" % args.gpus, "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.stdout.flush()
+    os.execv(sys.executable, cmd)
+
+
+def run_stub_replicas(args):
+    """The replica launch and aggregation path without a GPU (gloo): every rank pretends to have run K steps and the
+    job's figure is combined as for real replicas.  Exercised by the CPU tests."""
+    rank, world, local, dist = init_ranks("gloo")
+    K = args.steps
+    ms = 10.0 + 2.5 * rank                                # the slowest rank sets the job's time
+    nbytes = 4.0e9 * K
+    if dist:
+        dist.barrier()
+    ms_all, bytes_all, value = whole_job_throughput(dist, ms, nbytes, "cpu")
+    if rank == 0:
+        print(json.dumps({"metric": "prefix-hit KV fetch GB/s", "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": K,
+                          "warmup": args.warmup, "ms_per_step": round(ms_all / max(K, 1), 4), "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "u8", "data": "stub", "config": {"workload": "cpu_stub", "replicas": world}}), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_gpu(args):
+    import torch
+    rank, world, local, dist = init_ranks("nccl")
+    if world == 1:
         torch.cuda.set_device(0)
     from __graft_entry__ import build
     if rank == 0:
@@ -325,13 +374,14 @@ def run_gpu(args):
         ms = t0.elapsed_time(t1)
         s1 = wl.store.stats()
         fetched = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) + (s1.blocks_fetched[1] - s0.blocks_fetched[1])
-        moved = fetched + (s1.blocks_inserted - s0.blocks_inserted) + (s1.blocks_demoted - s0.blocks_demoted) + \
-            (s1.blocks_promoted - s0.blocks_promoted)
+        distinct = s1.blocks_fetched_distinct - s0.blocks_fetched_distinct
+        inserted, demoted, promoted = s1.blocks_inserted - s0.blocks_inserted, s1.blocks_demoted - s0.blocks_demoted, \
+            s1.blocks_promoted - s0.blocks_promoted
+        moved = fetched + inserted + demoted + promoted
         return dict(ms=ms, fetched=fetched, fetched_host=s1.blocks_fetched[1] - s0.blocks_fetched[1],
-                    inserted=s1.blocks_inserted - s0.blocks_inserted, demoted=s1.blocks_demoted - s0.blocks_demoted,
-                    host_dropped=s1.blocks_dropped[1] - s0.blocks_dropped[1], promoted=s1.blocks_promoted - s0.blocks_promoted,
-                    distinct=s1.blocks_fetched_distinct - s0.blocks_fetched_distinct,
-                    bytes=moved * block_rw, launches=wl.store.launch_count() - l0,
+                    inserted=inserted, demoted=demoted, host_dropped=s1.blocks_dropped[1] - s0.blocks_dropped[1], promoted=promoted,
+                    distinct=distinct, bytes=moved * block_rw, dram_bytes=(distinct + fetched + 2 * (inserted + demoted + promoted)) * wl.sh.block_bytes,
+                    launches=wl.store.launch_count() - l0,
                     probes=s1.probes_issued - s0.probes_issued, qblocks=s1.query_blocks - s0.query_blocks,
                     matched=s1.blocks_matched - s0.blocks_matched, dropped=s1.blocks_dropped[0] - s0.blocks_dropped[0])
 
@@ -341,15 +391,13 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    events = {"fetch": [], "insert": [], "evict": [], "promote": []}
+    events = {"fetch": [], "insert": [], "evict": [], "promote": [], "fetch_copy": [], "insert_copy": []}
     main = timed(i, K, False, events)
     clocks = sampler.stop() if rank == 0 else None
     i += K
     torch.cuda.synchronize()
-    fetch_ms = sum(a.elapsed_time(b) for a, b in events["fetch"])
-    insert_ms = sum(a.elapsed_time(b) for a, b in events["insert"])
-    evict_ms = sum(a.elapsed_time(b) for a, b in events["evict"])
-    promote_ms = sum(a.elapsed_time(b) for a, b in events["promote"])
+    ev_ms = {k: sum(a.elapsed_time(b) for a, b in v) for k, v in events.items()}
+    fetch_ms, insert_ms, evict_ms, promote_ms = ev_ms["fetch"], ev_ms["insert"], ev_ms["evict"], ev_ms["promote"]
     status = wl.store.status()
 
     e2e = None
@@ -365,59 +413,86 @@ def run_gpu(args):
         return reduce_over_ranks(dist, x, op, "cuda")
 
     MAX, SUM = "max", "sum"
-    ms, total_bytes, value = whole_job_throughput(dist, main["ms"], main["bytes"], "cuda")
+    ms, total_dram, value = whole_job_throughput(dist, main["ms"], main["dram_bytes"], "cuda")
+    delivered_all = agg(main["bytes"], SUM)
     peak, peak_kind = measured_peak()
-    fetch_bytes = main["fetched"] * block_rw
-    ach = fetch_bytes / (fetch_ms * 1e-3) / 1e9 if fetch_ms > 0 else 0.0
+    host_tier_fetch = bool(wl.host_blocks) or args.engine == "vector"
+    # the fetch copy kernel alone: bytes DRAM must move for it / its own duration
+    kern_ms = ev_ms["fetch_copy"] if ev_ms["fetch_copy"] > 0 else fetch_ms
+    fetch_dram = (main["distinct"] + main["fetched"]) * wl.sh.block_bytes
+    ach = fetch_dram / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
+    ach_delivered = main["fetched"] * block_rw / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
+    ins_kern_ms = ev_ms["insert_copy"]
     out = {
         "metric": "prefix-hit KV fetch GB/s", "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W_,
         "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8", "data": "synthetic",
         "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(getattr(wl.stream, "docs", ())) or wl.stream.n_conversations,
                    "batch": wl.batch, "eviction": args.policy, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
-                   "step": "lookup(PIN)+fetch+evict+insert+release", "fill_steps": n_fill, "replicas": world},
+                   "step": "lookup_fetch(PIN)+reserve+insert+release" if not (wl.promote or wl.async_demote) else "lookup(PIN)+promote+fetch+reserve+insert+release",
+                   "fill_steps": n_fill, "replicas": world},
+        "value_kind": "bytes DRAM must move (distinct source blocks read once + delivered blocks written + 2 x stored blocks) / step time",
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
-        # the same steps counted by the bytes DRAM has to move (a source block shared by several prompts is read once)
-        "value_on_needed_dram_bytes": round((main["distinct"] + main["fetched"] + 2 * (main["inserted"] + main["demoted"] + main["promoted"]))
-                                            * wl.sh.block_bytes / (main["ms"] * 1e-3) / 1e9, 1),
-        "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_inserted": main["inserted"] / K, "blocks_dropped": main["dropped"] / K,
+        # the same steps by the survey's convention: 2 x block bytes per delivered or stored block
+        "value_delivered_bytes": round(delivered_all / (ms * 1e-3) / 1e9, 1),
+        "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_fetched_distinct": main["distinct"] / K, "blocks_inserted": main["inserted"] / K,
+                     "blocks_dropped": main["dropped"] / K,
                      "hit_rate_blocks": round(main["matched"] / max(main["qblocks"], 1), 4),
-                     "fetch_call_ms": round(fetch_ms / K, 4), "insert_call_ms": round(insert_ms / K, 4),
-                     "insert_gbps": round(main["inserted"] * block_rw / max(insert_ms, 1e-9) / 1e6, 1),
+                     "fetch_call_ms": round(fetch_ms / K, 4), "fetch_copy_kernel_ms": round(ev_ms["fetch_copy"] / K, 4),
+                     "insert_call_ms": round(insert_ms / K, 4), "insert_copy_kernel_ms": round(ins_kern_ms / K, 4),
+                     "insert_copy_gbps": round(main["inserted"] * block_rw / max(ins_kern_ms, 1e-9) / 1e6, 1),
+                     "insert_call_gbps": round(main["inserted"] * block_rw / max(insert_ms, 1e-9) / 1e6, 1),
                      "lookup_probes": main["probes"] / K, "blocks_fetched_from_host": main["fetched_host"] / K,
                      "blocks_demoted": main["demoted"] / K, "host_blocks_dropped": main["host_dropped"] / K,
                      "evict_call_ms": round(evict_ms / K, 4), "blocks_promoted": main["promoted"] / K,
                      "promote_call_ms": round(promote_ms / K, 4),
-                     "demote_gbps_one_way": round(main["demoted"] * wl.sh.block_bytes / max(evict_ms, 1e-9) / 1e6, 1)},
+                     "demote_gbps_one_way": round(main["demoted"] * wl.sh.block_bytes / max(evict_ms, 1e-9) / 1e6, 1),
+                     "launches": main["launches"] / K},
         "gpu_launches": int(main["launches"]),
         "device_status": status,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "%s (ptstore_fetch)" % ("copy_vector_kernel<FETCH_MULTI>" if wl.host_blocks or args.engine == "vector" else "copy_bulk_multi_kernel"), "achieved": round(ach, 1), "peak": peak,
-                     "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": peak_kind + " (copy, read+write)",
+        "roofline": {"bound": "hbm", "kernel": "%s (gather of ptstore_lookup_fetch)" % ("copy_vector_kernel<FETCH_MULTI>" if host_tier_fetch else "copy_bulk_multi_kernel"),
+                     "achieved": round(ach, 1), "peak": peak, "unit": "GB/s", "frac": round(ach / peak, 4),
+                     "peak_kind": peak_kind + " (plain copy, read+write)",
+                     "achieved_kind": "bytes DRAM must move per launch (distinct source blocks read once + delivered blocks written) / kernel duration "
+                                      "(events recorded around the kernel by the library)",
                      "frac_of_nominal_8TBps": round(ach / NOMINAL_HBM_GBS, 4),
-                     "algorithmic_bytes_per_launch": fetch_bytes / K,
+                     "kernel_ms": round(kern_ms / K, 4),
+                     "dram_bytes_needed_per_launch": fetch_dram / K,
+                     "distinct_source_blocks_per_launch": main["distinct"] / K, "delivered_blocks_per_launch": main["fetched"] / K,
                      "traffic": args.traffic if args.traffic else round(
                          (NCU_READ_FACTOR * main["distinct"] + NCU_WRITE_FACTOR * main["fetched"]) * wl.sh.block_bytes / K),
-                     "traffic_kind": "ncu DRAM bytes per distinct block read and per block written (small-case capture, profiles/) "
-                                     "scaled by this launch's distinct source blocks and delivered blocks",
-                     "distinct_source_blocks_per_launch": main["distinct"] / K,
-                     "dram_bytes_needed_per_launch": (main["distinct"] + main["fetched"]) * wl.sh.block_bytes / K,
-                     "achieved_on_needed_dram_bytes": round((main["distinct"] + main["fetched"]) * wl.sh.block_bytes / max(fetch_ms, 1e-9) / 1e6, 1),
-                     "frac_on_needed_dram_bytes": round((main["distinct"] + main["fetched"]) * wl.sh.block_bytes / max(fetch_ms, 1e-9) / 1e6 / peak, 4),
-                     "note": "achieved counts 2 x block bytes per delivered block; a block named by several requests of the batch is "
-                             "read from DRAM once and written to each destination, so the DRAM traffic is below the algorithmic bytes "
-                             "and achieved can exceed the copy peak; the *_on_needed_dram_bytes figures use the bytes DRAM must move"},
+                     "traffic_kind": "modelled from the small-case ncu capture (profiles/): DRAM bytes per distinct block read and per block "
+                                     "written there, times this launch's distinct source blocks and delivered blocks",
+                     # the survey's convention (2 x block bytes per delivered block); above the copy peak because shared sources are read once
+                     "achieved_delivered_bytes": round(ach_delivered, 1), "frac_delivered_bytes": round(ach_delivered / peak, 4)},
     }
     if e2e:
         ems = agg(e2e["ms"], MAX)
-        eb = agg(e2e["bytes"], SUM)
+        eb = agg(e2e["dram_bytes"], SUM)
         if wl.host_blocks:
             out["host_link_gbps_measured"] = host_link_gbps(torch)
         out["e2e"] = {"value": round(eb / (ems * 1e-3) / 1e9, 1), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                      "ms_per_step": round(ems / K, 4)}
-    if rank == 0:
-        if world == 1 and not args.no_cpu:
+                      "ms_per_step": round(ems / K, 4), "launches_per_step": e2e["launches"] / K}
+    if world == 1 and rank == 0:
+        # free the serving store before the side records allocate theirs
+        wl.store.close()
+        wl.cache = None
+        wl.store = None
+        del wl
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+        if not args.no_latency and args.workload == "llama8b":
+            out["latency"] = latency_record(args, torch)
+            torch.cuda.empty_cache()
+        if not args.no_lookup and args.workload == "llama8b":
+            out["lookup"] = lookup_record(args, torch, K=args.lookup_calls, W_=5)["summary"]
+            torch.cuda.empty_cache()
+        if not args.no_cpu:
             out["cpu_baseline"] = cpu_oracle_sample(args)
+            out["cpu_baseline_all_threads"] = cpu_oracle_threads_sample(args)
+    if rank == 0:
         print(json.dumps(out), flush=True)
     if dist:
         dist.barrier()
@@ -454,13 +529,151 @@ def host_link_gbps(torch, gib=1):
     return out
 
 
-def run_lookup(args):
-    """configs[2]: lookup-only stress.  A step is one ptstore_lookup call over 16,384 requests x 64 blocks against a
-    10^6-node trie at load factor 0.7; K steps run back to back between two events."""
+# ---------------------------------------------------------------------------------------------------------
+def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, suffix_tokens=64, iters=40, headroom=64):
+    """Small batches, where the path is latency bound (the paper's end-to-end figure is the time to first token of one
+    request): every prompt is a stored 4k-token document (a full hit, 256 blocks = 512 MiB of KV) plus a fresh 64-token
+    question (4 new blocks), documents taken round robin so that no two prompts of a batch share one.  A step is
+    lookup_fetch(PIN) -> reserve -> insert -> release; the pool has little slack, so room has to be made all the time; a
+    reserve that must evict takes `headroom` blocks more than it needs, so most steps find room and skip the eviction.
+    Reported per batch size: microseconds of the whole step on the device (steps back to back, calls pre-marshalled), of a
+    step seen from the host (first call to the end of a synchronize), of each call, kernel launches per step, and the time
+    the step's copies would take at the measured copy bandwidth."""
+    import ctypes as C
+    from paper_2607_22648_b200 import binding as G
+    sh = W.LLAMA3_8B
+    B = sh.block_tokens
+    doc_blocks, suf_blocks = doc_tokens // B, suffix_tokens // B
+    mb = doc_blocks + suf_blocks
+    pool = n_docs * doc_blocks + 8 * n_docs * suf_blocks          # slack: suffixes of two rounds over the documents
+    bmax = max(batches)
+    st = G.PTStore(sh.layers, sh.heads, sh.dim, B, pool, max_requests=bmax, max_batch_blocks=bmax * mb)
+    cache = G.PagedKV(sh.layers, bmax * mb, sh.chunk_bytes)
+    rng = np.random.default_rng(W.BASE_SEED + 9)
+    docs = [rng.integers(0, 128256, size=doc_tokens, dtype=np.int32) for _ in range(n_docs)]
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    for t in cache.tensors:
+        t.random_(0, 256)
+    for k in range(0, n_docs, bmax):                                    # store the documents
+        part = docs[k:k + bmax]
+        toks, offs = W.ragged(part)
+        bt = np.arange(len(part) * mb, dtype=np.int32).reshape(len(part), mb)
+        st.insert(dev(toks), dev(offs), mb, cache, dev(bt))
+    assert st.status() == 0
+    peak, _ = measured_peak()
+    stream = torch.cuda.current_stream().cuda_stream
+    lib, h = G.lib, st.h
+    res = {}
+    next_doc = 0
+    for b in batches:
+        n_steps = 8 + 2 * iters
+        steps = []
+        for _ in range(n_steps):                                        # every step's inputs, resident on the device
+            seqs = []
+            for _r in range(b):
+                seqs.append(np.concatenate([docs[next_doc % n_docs], rng.integers(0, 128256, size=suffix_tokens, dtype=np.int32)]))
+                next_doc += 1
+            toks, offs = W.ragged(seqs)
+            bt = rng.permutation(b * mb).astype(np.int32).reshape(b, mb)
+            steps.append((dev(toks), dev(offs), dev(bt)))
+        matched = torch.empty(b, dtype=torch.int32, device="cuda")
+        ids = torch.empty((b, mb), dtype=torch.int32, device="cuda")
+        ins_ids = torch.empty((b, mb), dtype=torch.int32, device="cuda")
+        newb = torch.empty(b, dtype=torch.int32, device="cuda")
+        nev = torch.zeros(2, dtype=torch.int32, device="cuda")
+        cdesc = C.byref(cache.desc)
+
+        def calls(k):
+            t, o, bt = steps[k]
+            return [
+                ("lookup_fetch", lib.ptstore_lookup_fetch, (h, t.data_ptr(), o.data_ptr(), b, mb, G.PIN, cdesc, bt.data_ptr(), matched.data_ptr(), ids.data_ptr(), stream)),
+                ("reserve", lib.ptstore_reserve, (h, b * mb, headroom, matched.data_ptr(), b, 0, nev.data_ptr(), None, 0, stream)),
+                ("insert", lib.ptstore_insert, (h, t.data_ptr(), o.data_ptr(), b, mb, cdesc, bt.data_ptr(), ins_ids.data_ptr(), newb.data_ptr(), stream)),
+                ("release", lib.ptstore_release, (h, ids.data_ptr(), matched.data_ptr(), b, mb, stream)),
+            ]
+
+        k = 0
+        for _ in range(8):                                              # warm-up
+            for _n, f, a in calls(k):
+                assert f(*a) == 0
+            k += 1
+        torch.cuda.synchronize()
+        s0, l0 = st.stats(), st.launch_count()
+        # (a) steps back to back between two events
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            for _n, f, a in calls(k):
+                f(*a)
+            k += 1
+        e1.record(); torch.cuda.synchronize()
+        step_us = e0.elapsed_time(e1) / iters * 1e3
+        s1, l1 = st.stats(), st.launch_count()
+        # (b) one step at a time: per-call device time and the host's view (first call to end of synchronize)
+        per_call = {}
+        wall = []
+        for _ in range(iters):
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+            ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ca.record(); cb.record()                                    # bring the events into existence
+            lib.ptstore_time_next_copy(h, ca.cuda_event, cb.cuda_event)  # the gather kernel of the lookup_fetch below
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for q, (_n, f, a) in enumerate(calls(k)):
+                evs[q].record(); f(*a)
+            evs[4].record()
+            torch.cuda.synchronize()
+            wall.append((time.perf_counter() - t0) * 1e6)
+            for q, (n, _f, _a) in enumerate(calls(k)):
+                per_call.setdefault(n, []).append(evs[q].elapsed_time(evs[q + 1]) * 1e3)
+            per_call.setdefault("gather_kernel_of_lookup_fetch", []).append(ca.elapsed_time(cb) * 1e3)
+            k += 1
+        fetched = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) / iters
+        inserted = (s1.blocks_inserted - s0.blocks_inserted) / iters
+        dropped = (s1.blocks_dropped[0] - s0.blocks_dropped[0]) / iters
+        copy_bytes = (fetched + inserted) * 2 * sh.block_bytes
+        bound_us = copy_bytes / (peak * 1e9) * 1e6
+        res["batch%d" % b] = {"step_us": round(step_us, 1), "step_wall_us": round(float(np.median(wall)), 1),
+                              "call_us": {n: round(float(np.median(v)), 1) for n, v in per_call.items()},
+                              "launches_per_step": (l1 - l0) / iters, "blocks_fetched": fetched, "blocks_inserted": inserted,
+                              "blocks_evicted": dropped, "copy_bytes": copy_bytes, "copy_bound_us": round(bound_us, 1),
+                              "step_over_copy_bound": round(step_us / bound_us, 3), "gbps": round(copy_bytes / step_us / 1e3, 1)}
+    assert st.status() == 0
+    res["config"] = {"kv_shape": "32L x 8H x 128 bf16, block 16", "prompt": "%d-token stored document + %d fresh tokens" % (doc_tokens, suffix_tokens),
+                     "pool_blocks": pool, "docs": n_docs, "iters": iters, "reserve_headroom": headroom,
+                     "copy_bound": "bytes of the step's fetch and insert copies (read + write) / measured copy bandwidth"}
+    st.close()
+    return res
+
+
+def run_latency(args):
     import torch
     torch.cuda.set_device(0)
     from __graft_entry__ import build
     build()
+    sampler = ClockSampler(0)
+    sampler.start()
+    rec = latency_record(args, torch, iters=max(args.steps, 10))
+    clocks = sampler.stop()
+    b1 = rec["batch1"]
+    peak, kind = measured_peak()
+    out = {"metric": "prefix-hit KV fetch GB/s", "value": b1["gbps"], "unit": "GB/s", "n_gpus": 1, "steps": rec["config"]["iters"], "warmup": 8,
+           "ms_per_step": round(b1["step_us"] / 1e3, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+           "data": "synthetic", "config": dict(rec["config"], workload="latency_llama3_8b_4k_prompt_full_hit_batch1_4_16", l2="512 MiB of KV per prompt: larger than L2"),
+           "latency": rec, "gpu_launches": int(b1["launches_per_step"] * rec["config"]["iters"]), "clocks": clocks,
+           "roofline": {"bound": "hbm", "kernel": "whole batch-1 step", "achieved": b1["gbps"], "peak": peak, "unit": "GB/s",
+                        "frac": round(b1["gbps"] / peak, 4), "traffic": None, "peak_kind": kind + " (plain copy, read+write)"}}
+    print(json.dumps(out), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------------
+def lookup_record(args, torch, K=200, W_=5, variants=None):
+    """configs[2]: lookup-only stress.  One call = ptstore_lookup over 16,384 requests x 64 blocks against a 10^6-node trie at
+    load factor 0.7; K calls run back to back between two events (table and tokens warm in L2), then 10 more with L2
+    flushed before each."""
     from paper_2607_22648_b200 import binding as G
     ws = W.lookup_stress()
     wa = W.lookup_stress(all_hit=True)
@@ -479,10 +692,12 @@ def run_lookup(args):
     matched = torch.empty(16384, dtype=torch.int32, device="cuda")
     ids = torch.empty((16384, 64), dtype=torch.int32, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    K, W_ = args.steps, args.warmup
     sampler = ClockSampler(0)
-    for name, wl, flags in (("geometric_hit_depth", ws, 0), ("geometric_no_touch", ws, G.NO_TOUCH), ("geometric_pin", ws, G.PIN),
-                            ("all_hit", wa, G.NO_TOUCH)):
+    clocks = None
+    todo = (("geometric_hit_depth", ws, 0), ("geometric_no_touch", ws, G.NO_TOUCH), ("geometric_pin", ws, G.PIN), ("all_hit", wa, G.NO_TOUCH))
+    for name, wl, flags in todo:
+        if variants and name not in variants:
+            continue
         t, o = W.ragged(wl.queries)
         mb = W.max_blocks_of(wl.queries, 16)
         dt, do = dev(t), dev(o)
@@ -528,8 +743,27 @@ def run_lookup(args):
                      "query_blocks_per_s": round(q / (warm_ms * 1e-3)), "issued_probes_per_s": round(pr / (warm_ms * 1e-3)),
                      "matched_blocks_per_s": round((s1.blocks_matched - s0.blocks_matched) / K / (warm_ms * 1e-3)),
                      "issued_probes": pr, "query_blocks": q, "slots_per_probe": round((s1.slots_visited - s0.slots_visited) / K / max(pr, 1), 3),
-                     "launches": launches, "host_us_per_call": round(host_us, 2)}
+                     "launches": launches, "calls": K, "host_us_per_call": round(host_us, 2)}
     assert st.status() == 0
+    st.close()
+    main = res.get("geometric_hit_depth") or next(iter(res.values()))
+    summary = {"workload": "lookup_stress_1M_nodes_load0.7_16384x64_geometric0.9", "calls": K,
+               "query_blocks_per_s": main["query_blocks_per_s"], "issued_probes_per_s": main["issued_probes_per_s"],
+               "slots_per_probe": main["slots_per_probe"], "ms_warm": main["ms_warm"], "ms_l2_flushed": main["ms_l2_flushed"],
+               "l2_sectors_per_probe": L2_SECTORS_PER_PROBE, "l2_sectors_per_probe_kind": "modelled: from the ncu capture of this kernel in profiles/",
+               "all_hit_issued_probes_per_s": res["all_hit"]["issued_probes_per_s"] if "all_hit" in res else None,
+               "all_hit_ms_warm": res["all_hit"]["ms_warm"] if "all_hit" in res else None}
+    return {"variants": res, "summary": summary, "clocks": clocks}
+
+
+def run_lookup(args):
+    import torch
+    torch.cuda.set_device(0)
+    from __graft_entry__ import build
+    build()
+    K, W_ = args.steps, args.warmup
+    rec = lookup_record(args, torch, K, W_)
+    res = rec["variants"]
     main = res["geometric_hit_depth"]
     peak, kind = measured_peak()
     # algorithmic bytes of one call: tokens of the hashed blocks (64 B each), one 32-byte sector per probe, 4 B id per query block
@@ -539,7 +773,7 @@ def run_lookup(args):
            "data": "synthetic",
            "config": {"workload": "lookup_stress_1M_nodes_load0.7_16384x64_geometric0.9", "lanes_per_request": args.lanes or "auto",
                       "l2": "table (22.9 MB) is L2 resident by design; ms_l2_flushed gives the cold figure"},
-           "variants": res, "gpu_launches": main["launches"], "clocks": clocks,
+           "variants": res, "lookup": rec["summary"], "gpu_launches": main["launches"], "clocks": rec["clocks"],
            "roofline": {"bound": "hbm", "kernel": "lookup_kernel", "achieved": round(alg / (main["ms_warm"] * 1e-3) / 1e9, 1), "peak": peak,
                         "unit": "GB/s", "frac": round(alg / (main["ms_warm"] * 1e-3) / 1e9 / peak, 4), "traffic": None,
                         "note": "latency/issue bound, not bandwidth bound: the figure is context only"}}
@@ -585,6 +819,41 @@ def cpu_oracle_sample(args, steps=8, batch=8, pool_blocks=2800):
             "ms_per_step": round(t_total / steps * 1e3, 1), "host_cores_available": os.cpu_count()}
 
 
+def cpu_oracle_threads_sample(args, steps=8, batch=16, pool_blocks=2800):
+    """The oracle's read-only half of the step (lookup without stamps or pins, then the fetch) with the requests split
+    over every hardware thread; insert and eviction stay sequential and are not part of this figure."""
+    from oracle import Oracle
+    sh = W.LLAMA3_8B
+    stream = W.llama8b_stream(n_docs=args.docs or 500)
+    o = Oracle(sh.layers, sh.heads, sh.dim, sh.elem_bytes, sh.block_tokens, 0, pool_blocks, 0, byte_mode=True)
+    mb, B = stream.max_blocks, sh.block_tokens
+    rng = np.random.default_rng(6)
+    threads = os.cpu_count() or 1
+    batches = [stream.batch(batch)[0] for _ in range(steps + 1)]
+    need_max = max(sum(len(s) // B for s in b) for b in batches)
+    cache = o.new_cache(need_max + 1, fill=3)
+    moved, t_total = 0, 0.0
+    for k, seqs in enumerate(batches):
+        toks, offs = W.ragged(seqs)
+        bt = W.shuffled_block_tables(rng, seqs, B, mb, need_max + 1)
+        t0 = time.perf_counter()
+        m, ids = o.lookup_fetch_threads(toks, offs, mb, cache, bt, threads)
+        dt = time.perf_counter() - t0
+        short = sum(len(s) // B for s in seqs) - int(m.sum()) - o.free_count(0)
+        if short > 0:
+            o.evict(0, short, literal=False)
+        o.insert(toks, offs, mb, cache, bt)                # untimed: keeps the pool turning over as in the real step
+        if k == 0:
+            continue
+        t_total += dt
+        moved += int(m.sum()) * 2 * sh.block_bytes
+    o.close()
+    return {"value": round(moved / max(t_total, 1e-9) / 1e9, 2), "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": "lookup + fetch only (the read-only phases), %d steps of %d prompts of the same document stream split over %d "
+                      "threads, pool %d blocks" % (steps, batch, threads, pool_blocks),
+            "ms_per_step": round(t_total / steps * 1e3, 1)}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -611,26 +880,35 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--fill", type=int, default=6, help="untimed steps that fill the pool before warm-up")
-    ap.add_argument("--workload", default="llama8b", choices=["llama8b", "llama70b", "churn", "lookup", "multiturn"])
+    ap.add_argument("--workload", default="llama8b", choices=["llama8b", "llama70b", "churn", "lookup", "multiturn", "latency"])
     ap.add_argument("--block-tokens", type=int, default=0, help="llama8b workload: tokens per block (default 16)")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--docs", type=int, default=0)
     ap.add_argument("--pool-blocks", type=int, default=0)
     ap.add_argument("--host-gb", type=float, default=0.0)
     ap.add_argument("--policy", default="lru", choices=["lru", "gdsf"], help="eviction order")
-    ap.add_argument("--async-demote", action="store_true", help="churn workload: evict before fetch with ptstore_evict_async")
+    ap.add_argument("--async-demote", action="store_true", help="churn workload: reserve before fetch, demotion copy on the side stream")
     ap.add_argument("--promote", type=int, default=0, help="churn workload: host-tier blocks promoted into HBM per step (budget)")
     ap.add_argument("--lanes", type=int, default=0, help="lookup workload: lanes per request (0 = library default)")
+    ap.add_argument("--lookup-calls", type=int, default=200, help="back-to-back lookup calls of the lookup record")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-latency", action="store_true", help="skip the small-batch latency record")
+    ap.add_argument("--no-lookup", action="store_true", help="skip the lookup stress record")
+    ap.add_argument("--stub-cpu", action="store_true", help="replica launch and aggregation on CPU with a stub step (tests)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per fetch launch, if known (see profiles/)")
     args = ap.parse_args()
-    if args.warmup < 3 and args.impl == "ours":
-        args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        relaunch_as_replicas(args)                        # does not return
+    if args.stub_cpu:
+        run_stub_replicas(args)
     elif args.workload == "lookup":
         run_lookup(args)
+    elif args.workload == "latency":
+        run_latency(args)
     else:
         run_gpu(args)
 

@@ -282,14 +282,17 @@ int ptstore_evict_async(ptstore_t* st, int32_t tier, int32_t n_blocks, int32_t* 
  * Make room before a store, decided on the device (Section 1: blocks of finished requests are evicted when space is
  * needed; this is ptstore_evict(PTSTORE_TIER_HBM, n) with n computed where the free count lives, so the host need not
  * wait for a lookup's result before it can queue the eviction):
- *     n = max(0, want_free - sum(max(minus[i], 0), i < n_minus) - free HBM blocks),  capped at max_victims.
+ *     need = want_free - sum(max(minus[i], 0), i < n_minus) - free HBM blocks
+ *     n    = need > 0 ? need + headroom : 0,   capped at max_victims.
  * Typical use: want_free = full blocks of the batch, minus = the matched_blocks array the preceding lookup wrote.
+ * With headroom > 0 a call that has to evict takes that many blocks more, so that the calls after it find room and
+ * return at once (an eviction costs tens of microseconds whatever its size, which matters for small batches).
  *   flags       0, or PTSTORE_ASYNC_COPY (the demotion copy runs as in ptstore_evict_async; same ordering rules)
  *   n_evicted   out, device [2], as for ptstore_evict
  *   victim_ids  out, device [2*max_victims] or NULL (then max_victims is ignored), as for ptstore_evict
  * n_minus may not exceed max_requests (PTSTORE_E_LIMIT).
  */
-int ptstore_reserve(ptstore_t* st, int64_t want_free, const int32_t* minus, int32_t n_minus, uint32_t flags,
+int ptstore_reserve(ptstore_t* st, int64_t want_free, int32_t headroom, const int32_t* minus, int32_t n_minus, uint32_t flags,
                     int32_t* n_evicted, int32_t* victim_ids, int32_t max_victims, ptstore_stream_t stream);
 
 /* Make `stream` wait for a demotion copy left running by ptstore_evict_async (no-op if there is none). */

@@ -23,12 +23,14 @@
 // Pins (tests/test_oracle_*.py): longest-prefix result vs brute force over all stored sequences;
 // trie invariants; hash known answers, invertibility of mix and constants derived from sqrt/phi;
 // copies vs memcpy round trips with canaries; literal greedy eviction vs the sorted closed form;
-// allocation order closed form.  Parity unpinned: nothing exported here.
+// allocation order closed form; the threaded read-only pass vs the single-threaded functions.
+// Parity unpinned: nothing exported here.
 
 #include <cstdint>
 #include <cstring>
 #include <deque>
 #include <map>
+#include <thread>
 #include <algorithm>
 #include <tuple>
 #include <vector>
@@ -327,6 +329,50 @@ void oracle_fetch(void* h, const int32_t* ids, const int32_t* matched, int32_t R
           std::memcpy(layer_base[l] + s * kv_stride + (u64)db * block_stride,
                       src + ((u64)l * 2 + s) * o->chunk_bytes, o->chunk_bytes);
     }
+}
+
+// The two read-only phases (a lookup that neither stamps nor pins, then the fetch of what it matched) with the
+// requests split over `n_threads` host threads, each taking a contiguous range of requests.  It exists for the timed
+// CPU baseline only (what the same plain code does with every core of the machine); results are those of
+// oracle_lookup(NO_TOUCH) followed by oracle_fetch, which a test asserts.  The clock still advances by one.
+void oracle_lookup_fetch_threads(void* h, const int32_t* tokens, const int64_t* off, int32_t R, int32_t maxB,
+                                 uint8_t* const* layer_base, uint64_t kv_stride, uint64_t block_stride, uint32_t num_blocks,
+                                 const int32_t* bt, int32_t n_threads, int32_t* matched, int32_t* ids) {
+  Oracle* o = (Oracle*)h;
+  o->epoch += 1;
+  if (n_threads < 1) n_threads = 1;
+  std::vector<uint32_t> flagged((size_t)n_threads, 0);
+  auto work = [&](int t) {
+    const int r0 = (int)((int64_t)R * t / n_threads), r1 = (int)((int64_t)R * (t + 1) / n_threads);
+    for (int r = r0; r < r1; ++r) {
+      int nb = o->full_blocks(off, r, maxB);
+      const Node* cur = &o->root;
+      int m = 0;
+      for (; m < nb; ++m) {
+        const int32_t* tk = tokens + off[r] + (int64_t)m * o->B;
+        auto it = cur->children.find(std::vector<int32_t>(tk, tk + o->B));
+        if (it == cur->children.end()) break;
+        cur = it->second;
+        ids[(int64_t)r * maxB + m] = cur->block_id;
+      }
+      for (int j = m; j < maxB; ++j) ids[(int64_t)r * maxB + j] = -1;
+      matched[r] = m;
+      for (int j = 0; j < m; ++j) {
+        int32_t id = ids[(int64_t)r * maxB + j], db = bt[(int64_t)r * maxB + j];
+        if (db < 0 || (uint32_t)db >= num_blocks) { flagged[t] |= S_BOUNDS; continue; }
+        if (!o->byte_mode) continue;
+        const uint8_t* src = o->block_ptr(id);
+        for (int l = 0; l < o->layers; ++l)
+          for (int s = 0; s < 2; ++s)
+            std::memcpy(layer_base[l] + s * kv_stride + (u64)db * block_stride, src + ((u64)l * 2 + s) * o->chunk_bytes, o->chunk_bytes);
+      }
+    }
+  };
+  std::vector<std::thread> pool;
+  for (int t = 1; t < n_threads; ++t) pool.emplace_back(work, t);
+  work(0);
+  for (auto& th : pool) th.join();
+  for (uint32_t f : flagged) o->status |= f;
 }
 
 // sequential insert, request by request, block by block

@@ -25,7 +25,7 @@ def build_oracle(force=False):
     stamp = _LIB + ".srchash"
     if force or not os.path.exists(_LIB) or not os.path.exists(stamp) or open(stamp).read().strip() != want:
         tmp = _LIB + ".tmp%d" % os.getpid()
-        subprocess.check_call(["g++", "-std=c++17", "-O2", "-Wall", "-shared", "-fPIC", "-o", tmp, _SRC])
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-Wall", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC])
         os.replace(tmp, _LIB)
         with open(stamp, "w") as f:
             f.write(want)
@@ -49,6 +49,7 @@ def _load():
         lib.oracle_hash.argtypes = [vp, vp, vp, i32, i32, vp]
         lib.oracle_lookup.argtypes = [vp, vp, vp, i32, i32, C.c_uint32, vp, vp]
         lib.oracle_fetch.argtypes = [vp, vp, vp, i32, i32, vp, u64, u64, C.c_uint32, vp]
+        lib.oracle_lookup_fetch_threads.argtypes = [vp, vp, vp, i32, i32, vp, u64, u64, C.c_uint32, vp, i32, vp, vp]
         lib.oracle_insert.argtypes = [vp, vp, vp, i32, i32, vp, u64, u64, C.c_uint32, vp, vp, vp, vp]
         lib.oracle_release.argtypes = [vp, vp, vp, i32, i32]
         lib.oracle_evict.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -145,6 +146,17 @@ class Oracle:
         R, maxB = ids.shape
         keep, ptrs, kvs, bs, nb = self._cache_args(cache)
         self.lib.oracle_fetch(self.h, _p(ids), _p(matched), R, maxB, ptrs, kvs, bs, nb, _p(bt))
+
+    def lookup_fetch_threads(self, tokens, offsets, max_blocks, cache, block_tables, n_threads):
+        """Read-only lookup (no stamp, no pin) + fetch with the requests split over n_threads host threads."""
+        tokens, offsets, bt = _i32(tokens), np.ascontiguousarray(offsets, dtype=np.int64), _i32(block_tables)
+        R = len(offsets) - 1
+        matched = np.zeros(R, dtype=np.int32)
+        ids = np.zeros((R, max_blocks), dtype=np.int32)
+        keep, ptrs, kvs, bs, nb = self._cache_args(cache)
+        self.lib.oracle_lookup_fetch_threads(self.h, _p(tokens), _p(offsets), R, max_blocks, ptrs, kvs, bs, nb, _p(bt),
+                                             int(n_threads), _p(matched), _p(ids))
+        return matched, ids
 
     def insert(self, tokens, offsets, max_blocks, cache=None, block_tables=None, tags=None):
         tokens, offsets = _i32(tokens), np.ascontiguousarray(offsets, dtype=np.int64)

@@ -76,7 +76,7 @@ def _load():
     lib.ptstore_lookup.argtypes = [vp, vp, vp, i32, i32, u32, vp, vp, vp]
     lib.ptstore_fetch.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp]
     lib.ptstore_lookup_fetch.argtypes = [vp, vp, vp, i32, i32, u32, C.POINTER(PagedCache), vp, vp, vp, vp]
-    lib.ptstore_reserve.argtypes = [vp, C.c_int64, vp, i32, u32, vp, vp, i32, vp]
+    lib.ptstore_reserve.argtypes = [vp, C.c_int64, i32, vp, i32, u32, vp, vp, i32, vp]
     lib.ptstore_set_wait_limit.argtypes = [vp, u32]
     lib.ptstore_time_next_copy.argtypes = [vp, vp, vp]
     lib.ptstore_insert.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
@@ -230,13 +230,14 @@ class PTStore:
                                              _ptr(block_tables), _ptr(matched), _ptr(ids), _stream()), "ptstore_lookup_fetch")
         return matched, ids
 
-    def reserve(self, want_free, minus=None, flags=0, max_victims=0, n_evicted=None, victims=None):
-        """Evicts max(0, want_free - sum(minus) - free HBM blocks) blocks from HBM, decided on the device."""
+    def reserve(self, want_free, minus=None, flags=0, max_victims=0, n_evicted=None, victims=None, headroom=0):
+        """Evicts need + headroom blocks from HBM if need = want_free - sum(minus) - free HBM blocks is positive, decided on
+        the device."""
         if n_evicted is None:
             n_evicted = torch.zeros(2, dtype=torch.int32, device=self.device)
         if victims is None and max_victims:
             victims = torch.full((2 * max_victims,), -1, dtype=torch.int32, device=self.device)
-        self._check(lib.ptstore_reserve(self.h, int(want_free), _ptr(minus), minus.numel() if minus is not None else 0, flags,
+        self._check(lib.ptstore_reserve(self.h, int(want_free), int(headroom), _ptr(minus), minus.numel() if minus is not None else 0, flags,
                                         _ptr(n_evicted), _ptr(victims), max_victims, _stream()), "ptstore_reserve")
         return n_evicted, victims
 

@@ -62,6 +62,9 @@ struct Ctrl {
   // arrival counters of the grid-wide barriers of cooperative kernels: launch k uses entry k % BAR_SLOTS and zeroes
   // the entry half a ring ahead, so a counter is always zero when its turn comes, whatever happened to earlier launches
   u32 bar[64];
+#ifdef PTS_PHASE_TIMERS
+  u64 phase_ns[16];     // diagnostic build only: globaltimer at phase boundaries of the last cooperative kernel
+#endif
   // cumulative counters
   u64 query_blocks, probes_issued, slots_visited, blocks_matched;   // totals are these plus the stripes below
   u64 blocks_fetched[2];
@@ -232,6 +235,15 @@ __device__ __forceinline__ unsigned char* block_ptr(const Store& st, u32 id) {
 }
 
 __device__ __forceinline__ void raise(const Store& st, u32 bit) { atomicOr(&st.ctrl->status, bit); }
+
+#ifdef PTS_PHASE_TIMERS
+__device__ __forceinline__ void phase_mark(const Store& st, int i) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) { u64 t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); st.ctrl->phase_ns[i] = t; }
+}
+#define PHASE_MARK(st, i) phase_mark(st, i)
+#else
+#define PHASE_MARK(st, i)
+#endif
 
 // ---- grid-wide barrier for cooperative launches ---------------------------------------------------------------------
 // All CTAs of a cooperative launch are resident at once, so they may wait for one another.  Every CTA calls sync() the

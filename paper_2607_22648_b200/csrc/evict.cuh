@@ -30,7 +30,8 @@ constexpr int EV_WARPS = EV_THREADS / 32;
 struct EvictArgs {
   int tier;                 // tier the victims come from
   int mode;                 // EvictMode
-  // number of victims asked for: n, or (reserve form) max(0, want_free - sum(minus[0..n_minus)) - free blocks of tier 0)
+  // number of victims asked for: n; or (reserve form, want_free >= 0) need = want_free - sum(minus[0..n_minus)) - free
+  // blocks of tier 0, and need + n victims if need > 0, else none
   u32 n;
   long long want_free;      // < 0: plain form
   const int* minus;
@@ -116,6 +117,7 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
     long long need = a.want_free;
     for (int i = 0; i < a.n_minus; ++i) { int m = a.minus[i]; need -= m > 0 ? m : 0; }
     need -= (long long)count0;
+    if (need > 0) need += (long long)a.n;                 // short of room: evict `n` blocks more than needed right now
     n = need > 0 ? (need > 0x7FFFFFFFll ? 0x7FFFFFFFu : (u32)need) : 0u;
     if (n > a.max_victims) n = a.max_victims;
   }
@@ -128,6 +130,7 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
   u32 take = 0;
   int cur = 0;
 
+  PHASE_MARK(st, 0);
   if (want > 0) {
     // ---- host tier: which nodes are pinned in place by HBM descendants -------------------------------------------------
     const bool use_blocked = tier == 1 && st.n[1] > 0 && a.blocked != nullptr;
@@ -182,6 +185,7 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
       smax = x > smax ? x : smax; smin = y < smin ? y : smin; dmax = z > dmax ? z : dmax;
     }
     take = want < (u32)cand ? want : (u32)cand;
+    PHASE_MARK(st, 1);
 
     if (take > 0) {
       EvictPlan pl;
@@ -253,6 +257,7 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
         cur ^= 1;
       }
 
+      PHASE_MARK(st, 2);
       // ---- apply the first `take` records ------------------------------------------------------------------------------
       if (bar.ok) {
         const Key2* sorted = a.buf[cur];
@@ -296,6 +301,7 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
     }
   }
 
+  PHASE_MARK(st, 3);
   // ---- bookkeeping, by one thread.  Every CTA read the ring positions before its first barrier, or there was none ---------
   if (a.mode == EV_DEMOTE && a.victims && blockIdx.x == 0) {          // room-making drops are reported behind the demoted ids
     for (u32 i = threadIdx.x; i < host_dropped; i += EV_THREADS) a.victims[take + i] = a.room[i];

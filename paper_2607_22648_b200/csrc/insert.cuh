@@ -7,7 +7,7 @@
 //   rebuild : only when deleted table markers have piled up: move the table aside, clear it, put the
 //             live entries back.
 //   hash    : chained block keys (content hashes first, by one thread per block, when requests are few
-//             and long), and in the same sweep
+//             and long); serial along a request
 //   claim   : find the key of e in the table or claim an empty slot for it (atomicCAS on the key);
 //             every element that lands on a slot claimed in this call lowers slot.aux to its request
 //             index (atomicMin), so the lowest request presenting a new prefix becomes its creator.
@@ -53,18 +53,33 @@ __device__ __forceinline__ u32 block_scan_incl(u32 x, u32* warp_sums, u32* total
   return incl;
 }
 
-// find `key` or claim an empty slot for it; the lowest request index presenting a key claimed in this call owns it
+// find `key` or claim an empty slot for it; the lowest request index presenting a key claimed in this call owns it.
+// The probe run is read PROBE_WINDOW slots at a time (one round trip instead of four dependent ones).  Values read
+// early stay usable: during the claim phase a slot only ever changes from empty to a key, and an empty slot is never
+// passed over, it is claimed with a compare-and-swap whose result says what the slot really holds.
 __device__ __forceinline__ u32 claim_slot(const Store& st, u64 key, u32 r) {
   u64 s = home_slot(key, st.slots);
   u32 got = NO_SLOT;
-  for (u64 i = 0; i < st.slots; ++i) {
-    u64 k = *reinterpret_cast<volatile u64*>(&st.table[s].key);
-    if (k == KEY_EMPTY) {
-      k = atomicCAS(&st.table[s].key, KEY_EMPTY, key);
-      if (k == KEY_EMPTY) k = key;                     // claimed
+  for (u64 i = 0; i < st.slots && got == NO_SLOT; i += PROBE_WINDOW) {
+    u64 k[PROBE_WINDOW], idx[PROBE_WINDOW];
+#pragma unroll
+    for (int w = 0; w < PROBE_WINDOW; ++w) {
+      const u64 t = s + w;
+      idx[w] = t >= st.slots ? t - st.slots : t;
+      k[w] = *reinterpret_cast<volatile u64*>(&st.table[idx[w]].key);
     }
-    if (k == key) { got = (u32)s; break; }
-    s = (s + 1 == st.slots) ? 0 : s + 1;
+#pragma unroll
+    for (int w = 0; w < PROBE_WINDOW; ++w) {
+      if (got != NO_SLOT) break;
+      u64 kk = k[w];
+      if (kk == KEY_EMPTY) {
+        kk = atomicCAS(&st.table[idx[w]].key, KEY_EMPTY, key);
+        if (kk == KEY_EMPTY) kk = key;                 // claimed
+      }
+      if (kk == key) got = (u32)idx[w];
+    }
+    s += PROBE_WINDOW;
+    if (s >= st.slots) s -= st.slots;
   }
   if (got == NO_SLOT) { raise(st, S_TABLE_FULL); return got; }
   if (*reinterpret_cast<volatile u32*>(&st.table[got].id) == NO_ID) atomicMin(&st.table[got].aux, r);
@@ -106,8 +121,10 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
   const long long gthreads = (long long)gridDim.x * INS_THREADS;
   const long long gtid = (long long)blockIdx.x * INS_THREADS + threadIdx.x;
 
+  PHASE_MARK(st, 0);
   const bool rebuild = tomb0 > a.rebuild_threshold;
   if (rebuild) table_rebuild_coop(st, a.stash, bar);
+  PHASE_MARK(st, 1);
 
   // ---- hash + claim ----------------------------------------------------------------------------------------------------
   if (a.split) {
@@ -118,8 +135,11 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     }
     bar.sync(st);
   }
+  PHASE_MARK(st, 2);
   {
-    const long long warps = gthreads >> 5, warp0 = gtid >> 5;
+    // warp w of CTA b takes request groups w * gridDim + b, ...: consecutive groups go to different SMs, because a chain is
+    // a long dependent instruction sequence and many of them on one SM queue for its issue slots
+    const long long warps = gthreads >> 5, warp0 = (long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
     const long long groups = ((long long)a.R + G - 1) / G;
     for (long long grp = warp0; grp < groups && bar.ok; grp += warps) {
       const long long r = grp * G + sub;
@@ -135,19 +155,24 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
         if (active) cc = a.split ? a.keys[r * max_blocks + j] : content_block(a.tokens + tok0 + (long long)j * st.block_tokens, st.block_tokens);
         const int steps = most - base < L ? most - base : L;
         const u64 key = chain_chunk<L>(parent, cc, lane, steps);
-        if (active) {
-          a.keys[r * max_blocks + j] = key;
-          a.eslot[r * max_blocks + j] = claim_slot(st, key, (u32)r);
-        }
+        if (active) a.keys[r * max_blocks + j] = key;
         parent = __shfl_sync(FULL, key, (lane & ~(L - 1)) + L - 1);
       }
       if (valid) {
-        for (int j = nblk + sl; j < max_blocks; j += L) { a.keys[r * max_blocks + j] = 0; a.eslot[r * max_blocks + j] = NO_SLOT; }
+        for (int j = nblk + sl; j < max_blocks; j += L) a.keys[r * max_blocks + j] = 0;
         if (sl == 0) a.new_blocks[r] = 0;
       }
     }
   }
   bar.sync(st);
+  PHASE_MARK(st, 3);
+  // the chain is serial per request, the claims are not: one element per thread, so that the probe latencies overlap
+  for (long long e = gtid; e < total && bar.ok; e += gthreads) {
+    const u64 key = a.keys[e];
+    a.eslot[e] = key ? claim_slot(st, key, (u32)(e / max_blocks)) : NO_SLOT;
+  }
+  bar.sync(st);
+  PHASE_MARK(st, 4);
 
   // ---- count -----------------------------------------------------------------------------------------------------------
   const long long n_tiles = (total + INS_THREADS - 1) / INS_THREADS;
@@ -159,6 +184,7 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     if (threadIdx.x == 0) a.cta_sums[t] = sum;
   }
   bar.sync(st);
+  PHASE_MARK(st, 5);
 
   // ---- plan (the same in every CTA) and assign -------------------------------------------------------------------------
   u32 total_new;
@@ -222,7 +248,9 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     a.desc[rank] = d;
     atomicAdd(&a.new_blocks[e / max_blocks], 1);
   }
+  PHASE_MARK(st, 6);
   bar.sync(st);
+  PHASE_MARK(st, 7);
 
   // ---- finish ----------------------------------------------------------------------------------------------------------
   for (long long e = gtid; e < total && bar.ok; e += gthreads) {
@@ -234,6 +262,7 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     }
     a.ids_out[e] = out;
   }
+  PHASE_MARK(st, 8);
 }
 
 }  // namespace pts

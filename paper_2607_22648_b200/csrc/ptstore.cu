@@ -56,7 +56,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.ctrl = take(sizeof(Ctrl));
   L.blocked = take(N);
   // eviction: one sort record per block id of a tier, padded to whole tiles of the largest grid
-  const u64 recs = N + (u64)MAX_COOP_GRID * EV_THREADS;
+  const u64 recs = N + (u64)MAX_COOP_GRID * EV_THREADS + 8192;
   L.sort[0] = take(recs * sizeof(Key2)); L.sort[1] = take(recs * sizeof(Key2));
   L.hist = take((u64)256 * MAX_COOP_GRID * 4);
   L.tile_stats = take((u64)MAX_COOP_GRID * 4 * 8);
@@ -337,7 +337,10 @@ int join_tier(ptstore* h, cudaStream_t s) {
 // one phase of an eviction: a single cooperative launch
 int launch_evict(ptstore* h, int tier, int mode, EvictArgs a, cudaStream_t s) {
   const u32 span = tier ? h->cfg.host_blocks : h->cfg.hbm_blocks;
+  // CTAs: measured on B200, a pass over 512 records per CTA costs about as much as its two barriers, and barriers get
+  // slower with more CTAs: 512 records per CTA up to 64 CTAs, then 2048 per CTA up to one CTA per SM, then whatever it takes
   int grid = (int)((span + 511) / 512);
+  if (grid > 64) { grid = (int)((span + 2047) / 2048); if (grid < 64) grid = 64; }
   if (grid < 1) grid = 1;
   if (grid > h->coop_grid) grid = h->coop_grid;
   const u32 per = (span + grid - 1) / grid;
@@ -435,7 +438,13 @@ int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32
   if (split_path(h, R, max_blocks)) {
     int rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
     if (rc) return rc;
-    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, fl);
+    // few long requests: the chain loop of a warp is one long dependent sequence, so the lists are linked by a kernel of
+    // its own with one thread per entry rather than inside that loop (13 us against 4 us for one 260-block prompt)
+    FetchLink none = {};
+    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, none);
+    PTS_CHECK_LAUNCH(h);
+    if (!fl.bt) return PTSTORE_OK;
+    fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, block_ids, matched_blocks, R, max_blocks, fl);
     PTS_CHECK_LAUNCH(h);
     return PTSTORE_OK;
   }
@@ -692,12 +701,12 @@ int ptstore_evict_async(ptstore_t* h, int32_t tier, int32_t n_blocks, int32_t* n
   return evict_entry(h, tier, n_blocks, n_evicted, victim_ids, stream, true);
 }
 
-int ptstore_reserve(ptstore_t* h, int64_t want_free, const int32_t* minus, int32_t n_minus, uint32_t flags, int32_t* n_evicted,
-                    int32_t* victim_ids, int32_t max_victims, ptstore_stream_t stream) {
-  if (!h || want_free < 0 || n_minus < 0 || (n_minus > 0 && !minus) || !n_evicted || max_victims < 0) return PTSTORE_E_INVAL;
+int ptstore_reserve(ptstore_t* h, int64_t want_free, int32_t headroom, const int32_t* minus, int32_t n_minus, uint32_t flags,
+                    int32_t* n_evicted, int32_t* victim_ids, int32_t max_victims, ptstore_stream_t stream) {
+  if (!h || want_free < 0 || headroom < 0 || n_minus < 0 || (n_minus > 0 && !minus) || !n_evicted || max_victims < 0) return PTSTORE_E_INVAL;
   if ((u32)n_minus > h->cfg.max_requests) return PTSTORE_E_LIMIT;
   const u32 cap = victim_ids ? (u32)max_victims : 0x7FFFFFFFu;
-  return evict_impl(h, PTSTORE_TIER_HBM, 0, (long long)want_free, minus, n_minus, n_evicted, victim_ids, cap,
+  return evict_impl(h, PTSTORE_TIER_HBM, (u32)headroom, (long long)want_free, minus, n_minus, n_evicted, victim_ids, cap,
                     static_cast<cudaStream_t>(stream), (flags & PTSTORE_ASYNC_COPY) != 0);
 }
 
@@ -811,6 +820,14 @@ int ptstore_stats_enqueue(ptstore_t* h, ptstore_stats_t* out, ptstore_stream_t s
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
+
+#ifdef PTS_PHASE_TIMERS
+// diagnostic build only: copies the phase time stamps of the last cooperative kernel to the host (synchronises)
+extern "C" int ptstore_debug_phases(ptstore_t* h, uint64_t* out16) {
+  cudaDeviceSynchronize();
+  return cudaMemcpy(out16, h->st.ctrl->phase_ns, 16 * sizeof(uint64_t), cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : PTSTORE_E_CUDA;
+}
+#endif
 
 uint64_t ptstore_launch_count(const ptstore_t* h) { return h ? h->launches : 0; }
 int ptstore_last_cuda_error(const ptstore_t* h) { return h ? h->last_cuda : 0; }

@@ -67,13 +67,15 @@ class Pair:
             assert torch.equal(gc.tensors[l].cpu(), torch.from_numpy(np_cache[l])), "fetched bytes differ in layer %d" % l
         return mo, io
 
-    def reserve(self, want_free, minus, literal=True, asynchronous=False, max_victims=None):
+    def reserve(self, want_free, minus, literal=True, asynchronous=False, max_victims=None, headroom=0):
         """ptstore_reserve against the oracle's evict of the count the definition gives."""
-        n = max(0, int(want_free) - int(np.maximum(minus, 0).sum()) - self.o.free_count(0))
+        n = int(want_free) - int(np.maximum(minus, 0).sum()) - self.o.free_count(0)
+        n = n + headroom if n > 0 else 0
         cap = n if max_victims is None else max_victims
         n = min(n, cap)
         ne_o, v_o = self.o.evict(0, n, literal=literal)
-        ne_g, v_g = self.g.reserve(want_free, dev(minus.astype(np.int32)), G.ASYNC_COPY if asynchronous else 0, max_victims=max(cap, 1))
+        ne_g, v_g = self.g.reserve(want_free, dev(minus.astype(np.int32)), G.ASYNC_COPY if asynchronous else 0, max_victims=max(cap, 1),
+                                   headroom=headroom)
         ne_g = ne_g.cpu().numpy()
         assert ne_o.tolist() == ne_g.tolist(), ("evicted counts differ", ne_o, ne_g)
         k = int(ne_o.sum())

@@ -705,7 +705,8 @@ def test_fused_step_lockstep(host, policy):
             dst = W.random_kv_cache(seed * 1000 + step, sh, nd)          # holds the new blocks' K/V; hits overwrite their part
             mo, io = p.lookup_fetch(batch, mb, dst, bt, flags=1)
             asyn = bool(host) and step % 3 == 0
-            p.reserve(sum(upper), mo, literal=bool(step % 2), asynchronous=asyn, max_victims=40 if step % 5 else 3)
+            p.reserve(sum(upper), mo, literal=bool(step % 2), asynchronous=asyn, max_victims=40 if step % 5 else 3,
+                      headroom=(0, 0, 5)[step % 3])
             p.insert(batch, mb, dst, bt)
             p.release(io, mo)
             p.check_status()

@@ -53,3 +53,18 @@ def test_reference_arm_prints_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_that_many_replicas():
+    """`bench.py --gpus 2` outside any launcher must itself start two ranks (here with the CPU stub of the step and
+    gloo) and report n_gpus 2, the slowest rank's time and the sum of the work."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub-cpu", "--steps", "4", "--warmup", "0"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["config"]["replicas"] == 2
+    assert out["ms_per_step"] == 12.5 / 4                      # max over ranks of 10.0 and 12.5 ms
+    assert abs(out["value"] - 2 * 4.0e9 * 4 / 12.5e-3 / 1e9) < 0.1

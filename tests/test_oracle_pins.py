@@ -687,3 +687,32 @@ def test_chained_keys_spread_evenly_over_a_table():
     expect = slots * (1 - np.exp(-50000 / slots))                      # balls into bins
     assert abs(occupied - expect) / expect < 0.01
     assert np.bincount(home, minlength=slots).max() <= 8
+
+
+def test_threaded_read_only_pass_equals_the_single_threaded_functions():
+    """The baseline's all-cores variant (lookup without stamps or pins + fetch, requests split over threads) against the
+    plain functions on the tiny config, for several thread counts including more threads than requests."""
+    w = W.tiny()
+    sh, B = w.shape, w.shape.block_tokens
+    rng = np.random.default_rng(3)
+    o = Oracle(sh.layers, sh.heads, sh.dim, sh.elem_bytes, B, 0, w.pool_blocks)
+    smb = W.max_blocks_of(w.store_seqs, B)
+    need = sum(len(s) // B for s in w.store_seqs)
+    o.insert(*W.ragged(w.store_seqs), smb, W.random_kv_cache(1, sh, need), W.shuffled_block_tables(rng, w.store_seqs, B, smb, need))
+    batch = w.queries + w.store_seqs[:9]
+    mb = W.max_blocks_of(batch, B)
+    toks, offs = W.ragged(batch)
+    nd = sum(len(s) // B for s in batch) + 3
+    bt = W.shuffled_block_tables(rng, batch, B, mb, nd)
+    m0, i0 = o.lookup(toks, offs, mb, NO_TOUCH)
+    want = o.new_cache(nd, fill=9)
+    o.fetch(i0, m0, want, bt)
+    stamps = [o.block_info(i)["last_use"] for i in range(64)]
+    for threads in (1, 2, 5, 64):
+        got = o.new_cache(nd, fill=9)
+        e0 = o.epoch()
+        m, ids = o.lookup_fetch_threads(toks, offs, mb, got, bt, threads)
+        assert (m == m0).all() and (ids == i0).all() and o.epoch() == e0 + 1
+        for l in range(sh.layers):
+            assert (got[l] == want[l]).all()
+    assert stamps == [o.block_info(i)["last_use"] for i in range(64)] and o.status() == 0
