@@ -238,7 +238,7 @@ class Serving:
         a = self._ev() if timed else None
         if timed:
             self._time_copy(events["insert_copy"])
-        st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb)
+        st.insert(d["tokens"], d["offsets"], self.mb, self.cache, d["bt"], self.ins_ids, self.newb, after_lookup=True)
         if timed:
             events["insert"].append((a, self._ev()))
         st.release(self.ids, self.matched)
@@ -429,7 +429,7 @@ def run_gpu(args):
         "dtype": "u8", "data": "synthetic",
         "config": {"workload": wl.name, "kv_shape": wl.kv, "pool_blocks": wl.pool_blocks, "host_blocks": wl.host_blocks, "docs": len(getattr(wl.stream, "docs", ())) or wl.stream.n_conversations,
                    "batch": wl.batch, "eviction": args.policy, "engine": args.engine, "variant": args.variant, "l2": "inputs larger than L2 (>= 20 GB per step)",
-                   "step": "lookup_fetch(PIN)+reserve+insert+release" if not (wl.promote or wl.async_demote) else "lookup(PIN)+promote+fetch+reserve+insert+release",
+                   "step": "lookup_fetch(PIN)+reserve+insert_after_lookup+release" if not (wl.promote or wl.async_demote) else "lookup(PIN)+promote+fetch+reserve+insert+release",
                    "fill_steps": n_fill, "replicas": world},
         "value_kind": "bytes DRAM must move (distinct source blocks read once + delivered blocks written + 2 x stored blocks) / step time",
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
@@ -486,6 +486,10 @@ def run_gpu(args):
         if not args.no_latency and args.workload == "llama8b":
             out["latency"] = latency_record(args, torch)
             torch.cuda.empty_cache()
+        if not args.no_ceilings and args.workload == "llama8b":
+            ratio = main["fetched"] / max(main["distinct"], 1)
+            out["copy_engine_ceilings"] = ceilings_record(torch, writes_x100=int(round(ratio * 100)))
+            torch.cuda.empty_cache()
         if not args.no_lookup and args.workload == "llama8b":
             out["lookup"] = lookup_record(args, torch, K=args.lookup_calls, W_=5)["summary"]
             torch.cuda.empty_cache()
@@ -534,7 +538,7 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
     """Small batches, where the path is latency bound (the paper's end-to-end figure is the time to first token of one
     request): every prompt is a stored 4k-token document (a full hit, 256 blocks = 512 MiB of KV) plus a fresh 64-token
     question (4 new blocks), documents taken round robin so that no two prompts of a batch share one.  A step is
-    lookup_fetch(PIN) -> reserve -> insert -> release; the pool has little slack, so room has to be made all the time; a
+    lookup_fetch(PIN) -> reserve -> insert_after_lookup -> release; the pool has little slack, so room has to be made all the time; a
     reserve that must evict takes `headroom` blocks more than it needs, so most steps find room and skip the eviction.
     Reported per batch size: microseconds of the whole step on the device (steps back to back, calls pre-marshalled), of a
     step seen from the host (first call to the end of a synchronize), of each call, kernel launches per step, and the time
@@ -591,7 +595,7 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
             return [
                 ("lookup_fetch", lib.ptstore_lookup_fetch, (h, t.data_ptr(), o.data_ptr(), b, mb, G.PIN, cdesc, bt.data_ptr(), matched.data_ptr(), ids.data_ptr(), stream)),
                 ("reserve", lib.ptstore_reserve, (h, b * mb, headroom, matched.data_ptr(), b, 0, nev.data_ptr(), None, 0, stream)),
-                ("insert", lib.ptstore_insert, (h, t.data_ptr(), o.data_ptr(), b, mb, cdesc, bt.data_ptr(), ins_ids.data_ptr(), newb.data_ptr(), stream)),
+                ("insert", lib.ptstore_insert_after_lookup, (h, t.data_ptr(), o.data_ptr(), b, mb, cdesc, bt.data_ptr(), ins_ids.data_ptr(), newb.data_ptr(), stream)),
                 ("release", lib.ptstore_release, (h, ids.data_ptr(), matched.data_ptr(), b, mb, stream)),
             ]
 
@@ -647,6 +651,45 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
                      "copy_bound": "bytes of the step's fetch and insert copies (read + write) / measured copy bandwidth"}
     st.close()
     return res
+
+
+def ceilings_record(torch, writes_x100=274, gib=4):
+    """What the bulk copy engine itself reaches on this GPU, by traffic pattern (ptstore_copy_probe over plain buffers larger
+    than L2, the ring the store uses for 32 KiB chunks, best of 4 launches each): loads only, stores only, a 1:1 copy, and
+    the read-once-write-many mix of the benchmark's fetch."""
+    from paper_2607_22648_b200 import binding as G
+    n = gib << 30
+    w = (writes_x100 + 99) // 100
+    src = torch.empty(n, dtype=torch.uint8, device="cuda").fill_(3)
+    dst = torch.empty(n * w, dtype=torch.uint8, device="cuda").fill_(5)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = {}
+    for name, mode, moved in (("read_only", G.PROBE_READ, n), ("write_only", G.PROBE_WRITE, n), ("copy_1to1", G.PROBE_COPY, 2 * n),
+                              ("mix_1to%.2f" % (writes_x100 / 100), G.PROBE_MIX, n + n * writes_x100 / 100)):
+        best = 1e9
+        for r in range(5):
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            G.copy_probe(src, dst, n, mode, writes_x100, status=status)
+            b.record(); torch.cuda.synchronize()
+            if r:
+                best = min(best, a.elapsed_time(b))
+        out[name] = round(moved / (best * 1e-3) / 1e9, 1)
+    # the same 1:1 copy with four stages: more loads in flight help the loads and cost the copy
+    for name, mode, moved in (("read_only_4_stages", G.PROBE_READ, n), ("copy_1to1_4_stages", G.PROBE_COPY, 2 * n)):
+        best = 1e9
+        for r in range(4):
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            G.copy_probe(src, dst, n, mode, writes_x100, stages=4, status=status)
+            b.record(); torch.cuda.synchronize()
+            if r:
+                best = min(best, a.elapsed_time(b))
+        out[name] = round(moved / (best * 1e-3) / 1e9, 1)
+    assert int(status.item()) == 0
+    out["unit"] = "GB/s (bytes read + bytes written)"
+    out["how"] = "ptstore_copy_probe, 3 stages x 32 KiB, 1 CTA per SM, %d GiB read per launch, paged-cache-like destinations" % gib
+    return out
 
 
 def run_latency(args):
@@ -895,6 +938,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-latency", action="store_true", help="skip the small-batch latency record")
     ap.add_argument("--no-lookup", action="store_true", help="skip the lookup stress record")
+    ap.add_argument("--no-ceilings", action="store_true", help="skip the copy-engine ceiling probes")
     ap.add_argument("--stub-cpu", action="store_true", help="replica launch and aggregation on CPU with a stub step (tests)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per fetch launch, if known (see profiles/)")
     args = ap.parse_args()

@@ -238,6 +238,22 @@ int ptstore_insert(ptstore_t* st, const int32_t* tokens, const int64_t* offsets,
                    int32_t* block_ids, int32_t* new_blocks, ptstore_stream_t stream);
 
 /*
+ * ptstore_insert for the batch the handle's most recent ptstore_lookup / ptstore_lookup_fetch call was given (Section 4:
+ * a store begins by finding the longest common prefix, which the preceding load has just done for the same prompt).
+ * Same results as ptstore_insert in every case.  If tokens, offsets, R and max_blocks are those of that lookup - the same
+ * pointers and sizes, and the caller has not changed the arrays' contents since - and requests are few and long (a warp per
+ * request: fewer than 1024 requests of more than 16 blocks), the chained block keys that lookup computed are reused and
+ * hashing resumes behind them; the hash chain of a long prompt is a serial computation, so this takes tens of microseconds
+ * off a small batch.  Otherwise the call is ptstore_insert.
+ */
+int ptstore_insert_after_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                                const ptstore_paged_cache_t* src /*host struct*/, const int32_t* block_tables,
+                                int32_t* block_ids, int32_t* new_blocks, ptstore_stream_t stream);
+
+/* Calls of ptstore_insert_after_lookup so far that did reuse a lookup's keys (host counter, no sync). */
+uint64_t ptstore_resumed_inserts(const ptstore_t* st);
+
+/*
  * Drop one reference per (r, j < matched_blocks[r]) pair (the counterpart of PIN; Section 1: blocks
  * of finished requests become evictable).  A count that is already zero stays zero and raises S_STATE.
  */
@@ -350,6 +366,28 @@ int ptstore_set_wait_limit(ptstore_t* st, uint32_t polls);
  * which is what a bandwidth figure for the copy engine has to be divided by.
  */
 int ptstore_time_next_copy(ptstore_t* st, void* before /*cudaEvent_t*/, void* after /*cudaEvent_t*/);
+
+/*
+ * Measurement aid (no paper counterpart; needs no handle): run the bulk copy engine's ring over two plain device buffers
+ * in one traffic pattern, so the ceilings of the engine on this GPU can be measured next to a real fetch.
+ *   mode  PTSTORE_PROBE_READ   loads only (global -> shared, data dropped)
+ *         PTSTORE_PROBE_WRITE  stores only (shared -> global from a resident stage)
+ *         PTSTORE_PROBE_COPY   one store per load
+ *         PTSTORE_PROBE_MIX    writes_x100 / 100 stores per load on average (100..3200): the pattern of a fetch whose source
+ *                              blocks are shared by several prompts
+ *   src   `bytes` bytes; dst: `bytes` * ceil(writes_x100 / 100) bytes (`bytes` for the other modes); both 16-byte aligned
+ *   bytes a multiple of 1024 * stage_bytes; with scatter != 0, bytes / stage_bytes / 64 must be a power of two
+ *   stages, stage_bytes, ctas_per_sm   the ring: 2..32 stages of stage_bytes (multiple of 16, ring <= 200 KiB), 1..8 CTAs per SM
+ *   scatter != 0   destinations laid out like a paged cache (64 planes, a pseudo-random block per 64 pieces) instead of linearly
+ *   status device uint32, caller-cleared: PTSTORE_S_TIMEOUT is OR-ed in if a bounded wait expired
+ * Bytes moved: `bytes` read (not for WRITE) + `bytes` x stores per load written.  Enqueues one kernel on `stream`.
+ */
+#define PTSTORE_PROBE_READ   0
+#define PTSTORE_PROBE_WRITE  1
+#define PTSTORE_PROBE_COPY   2
+#define PTSTORE_PROBE_MIX    3
+int ptstore_copy_probe(const void* src, void* dst, uint64_t bytes, int32_t mode, uint32_t writes_x100, int32_t stages,
+                       uint32_t stage_bytes, int32_t ctas_per_sm, int32_t scatter, uint32_t* status, ptstore_stream_t stream);
 
 /* Number of this library's kernels launched through the handle so far (host counter, no sync). */
 uint64_t ptstore_launch_count(const ptstore_t* st);

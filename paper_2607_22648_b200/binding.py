@@ -59,7 +59,8 @@ class Stats(C.Structure):
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",
            "ptstore_fetch", "ptstore_insert", "ptstore_release", "ptstore_evict", "ptstore_status", "ptstore_stats",
            "ptstore_launch_count", "ptstore_last_cuda_error", "ptstore_strerror", "ptstore_fetch_static", "ptstore_promote", "ptstore_evict_async", "ptstore_join", "ptstore_stats_enqueue", "ptstore_lookup_fetch",
-           "ptstore_reserve", "ptstore_set_wait_limit", "ptstore_time_next_copy"]
+           "ptstore_reserve", "ptstore_set_wait_limit", "ptstore_time_next_copy", "ptstore_copy_probe",
+           "ptstore_insert_after_lookup", "ptstore_resumed_inserts"]
 
 
 def _load():
@@ -79,7 +80,11 @@ def _load():
     lib.ptstore_reserve.argtypes = [vp, C.c_int64, i32, vp, i32, u32, vp, vp, i32, vp]
     lib.ptstore_set_wait_limit.argtypes = [vp, u32]
     lib.ptstore_time_next_copy.argtypes = [vp, vp, vp]
+    lib.ptstore_copy_probe.argtypes = [vp, vp, u64, i32, u32, i32, u32, i32, i32, vp, vp]
     lib.ptstore_insert.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
+    lib.ptstore_insert_after_lookup.argtypes = [vp, vp, vp, i32, i32, C.POINTER(PagedCache), vp, vp, vp, vp]
+    lib.ptstore_resumed_inserts.restype = u64
+    lib.ptstore_resumed_inserts.argtypes = [vp]
     lib.ptstore_release.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.ptstore_evict.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.ptstore_evict_async.argtypes = [vp, i32, i32, vp, vp, vp]
@@ -126,6 +131,20 @@ class PagedKV:
         t0 = self.tensors[0]
         self.desc = PagedCache(self.ptrs.data_ptr(), t0.stride(0) * t0.element_size(), t0.stride(1) * t0.element_size(),
                                num_blocks, 0)
+
+
+PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MIX = 0, 1, 2, 3
+
+
+def copy_probe(src, dst, nbytes, mode, writes_x100=100, stages=3, stage_bytes=32768, ctas_per_sm=1, scatter=True, status=None):
+    """ptstore_copy_probe: one launch of the bulk copy ring over plain buffers (uint8 device tensors) in one traffic pattern."""
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=src.device)
+    rc = lib.ptstore_copy_probe(_ptr(src), _ptr(dst), nbytes, mode, writes_x100, stages, stage_bytes, ctas_per_sm, 1 if scatter else 0,
+                                _ptr(status), _stream())
+    if rc:
+        raise PTStoreError(rc, "ptstore_copy_probe")
+    return status
 
 
 STATIC_MAX_REQUESTS, STATIC_MAX_PAIRS = 1024, 65536
@@ -248,16 +267,21 @@ class PTStore:
     def set_wait_limit(self, polls):
         self._check(lib.ptstore_set_wait_limit(self.h, polls), "ptstore_set_wait_limit")
 
-    def insert(self, tokens, offsets, max_blocks, cache=None, block_tables=None, ids=None, new_blocks=None):
+    def insert(self, tokens, offsets, max_blocks, cache=None, block_tables=None, ids=None, new_blocks=None, after_lookup=False):
+        """after_lookup: ptstore_insert_after_lookup (reuses the keys of the last lookup if it saw these very tensors)."""
         R = offsets.numel() - 1
         if ids is None:
             ids = torch.empty((R, max_blocks), dtype=torch.int32, device=self.device)
         if new_blocks is None:
             new_blocks = torch.empty(R, dtype=torch.int32, device=self.device)
         desc = C.byref(cache.desc) if cache is not None else None
-        self._check(lib.ptstore_insert(self.h, _ptr(tokens), _ptr(offsets), R, max_blocks, desc, _ptr(block_tables),
-                                       _ptr(ids), _ptr(new_blocks), _stream()), "ptstore_insert")
+        fn = lib.ptstore_insert_after_lookup if after_lookup else lib.ptstore_insert
+        self._check(fn(self.h, _ptr(tokens), _ptr(offsets), R, max_blocks, desc, _ptr(block_tables),
+                       _ptr(ids), _ptr(new_blocks), _stream()), "ptstore_insert")
         return ids, new_blocks
+
+    def resumed_inserts(self):
+        return int(lib.ptstore_resumed_inserts(self.h))
 
     def release(self, ids, matched):
         R, mb = ids.shape

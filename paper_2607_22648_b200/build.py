@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libptstore.so")
-SOURCES = ["ptstore.cu", "fetch_static.cu"]
+SOURCES = ["ptstore.cu", "fetch_static.cu", "copy_probe.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fPIC",
               "-shared", "-cudart", "shared"]
 

@@ -14,7 +14,8 @@
 //   - every call on a GPU shares the one array.  Calls that overlap on the GPU (two streams, two
 //     threads) race on it; serialise them;
 //   - the first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
-//     device current; make that first call before any stream capture begins;
+//     device current; make that first call before any stream capture begins, and not from two host threads
+//     at once (the address is cached without a lock);
 //   - nothing is allocated or freed here: no cudaMalloc, no cudaFree, no allocating library call.
 #include "../../include/ptstore.h"
 
@@ -100,14 +101,19 @@ extern "C" int ptstore_fetch_static(const void* hbm_pool, uint32_t hbm_blocks, u
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) { (void)cudaGetLastError(); return PTSTORE_E_CUDA; }
 
+  (void)cudaGetLastError();                                   // an error left pending by the caller's earlier calls is not ours to report
   static_begin_kernel<<<1, 1, 0, s>>>(st.ctrl);              // the array keeps the last call's contents: clear what must start at zero
+  if (cudaGetLastError() != cudaSuccess) return PTSTORE_E_CUDA;
   if (R > 0) {
     scan_matched_kernel<<<1, 1024, 0, s>>>(st, matched_blocks, R, max_blocks, prefix);
+    if (cudaGetLastError() != cudaSuccess) return PTSTORE_E_CUDA;
     long long total = (long long)R * max_blocks;
     int grid = (int)((total + 255) / 256);
     if (grid > sms * 8) grid = sms * 8;
     build_pairs_kernel<<<grid, 256, 0, s>>>(st, block_ids, matched_blocks, block_tables, R, max_blocks, dst->num_blocks, prefix, desc);
+    if (cudaGetLastError() != cudaSuccess) return PTSTORE_E_CUDA;
     copy_vector_kernel<COPY_FETCH, 256, 4><<<sms * 16, 256, 0, s>>>(st, pc, desc, &st.ctrl->n_pairs);
+    if (cudaGetLastError() != cudaSuccess) return PTSTORE_E_CUDA;
   }
   static_end_kernel<<<1, 1, 0, s>>>(st.ctrl, status_out);
   if (cudaGetLastError() != cudaSuccess) return PTSTORE_E_CUDA;

@@ -91,6 +91,8 @@ struct InsertArgs {
   const long long* offsets;
   int R, max_blocks;
   int split;                // 1: content hashes first, one thread per block (few long requests); needs L == 32
+  const u32* hashed;        // non-null (L == 32 only): keys[r][0 .. hashed[r]) already hold the chained keys of request r,
+                            // left there by the lookup of the same batch; hashing resumes behind them
   u64* keys;                // scratch [R*max_blocks]
   u32* eslot;               // scratch [R*max_blocks]
   u32* cta_sums;            // scratch [tiles]
@@ -130,7 +132,7 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
   if (a.split) {
     for (long long e = gtid; e < total; e += gthreads) {
       const int r = (int)(e / max_blocks), j = (int)(e % max_blocks);
-      if (j < full_blocks(a.offsets, r, st.block_tokens, max_blocks))
+      if (j < full_blocks(a.offsets, r, st.block_tokens, max_blocks) && !(a.hashed && (u32)j < a.hashed[r]))
         a.keys[e] = content_block(a.tokens + a.offsets[r] + (long long)j * st.block_tokens, st.block_tokens);
     }
     bar.sync(st);
@@ -148,7 +150,13 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
       const long long tok0 = valid ? a.offsets[r] : 0;
       u64 parent = st.root_key;
       const int most = __reduce_max_sync(FULL, nblk);
-      for (int base = 0; base < most; base += L) {
+      int base0 = 0;
+      if (L == 32 && a.hashed && valid) {               // a warp per request: resume behind the keys the lookup left
+        const int have = (int)a.hashed[r];
+        base0 = have < nblk ? have : nblk;              // a multiple of 32, or all of the request
+        if (base0 > 0) parent = a.keys[r * max_blocks + base0 - 1];
+      }
+      for (int base = base0; base < most; base += L) {
         const int j = base + sl;
         const bool active = j < nblk;
         u64 cc = 0;

@@ -128,7 +128,8 @@ template <int L>
 __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __restrict__ tokens,
                                                      const long long* __restrict__ offsets, int R, int max_blocks,
                                                      u32 flags, u64 epoch, int* __restrict__ matched,
-                                                     int* __restrict__ ids_out, FetchLink fl) {
+                                                     int* __restrict__ ids_out, FetchLink fl, u64* __restrict__ keys_out,
+                                                     u32* __restrict__ hashed) {
   constexpr int G = 32 / L;
   constexpr unsigned SUBMASK = (L == 32) ? FULL : ((1u << L) - 1u);
   const int lane = threadIdx.x & 31, sl = lane & (L - 1), sub = lane / L;
@@ -143,6 +144,7 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
   bool done = nblk == 0;
   u32 my_probes = 0, my_visited = 0;
   u32 cnt0 = 0, cnt1 = 0;
+  int n_hashed = 0;
   if (fl.bt && blockIdx.x == 0 && threadIdx.x == 0) link_prepare_next(st, fl);
 
   for (int base = 0;; base += L) {
@@ -154,6 +156,8 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
     const int left = done ? 0 : (nblk - base < L ? nblk - base : L);
     const int steps = __reduce_max_sync(FULL, left);
     const u64 key = chain_chunk<L>(parent, c, lane, steps);
+    if (active) keys_out[r * max_blocks + j] = key;              // kept for an insert of the same batch
+    if (!done) n_hashed = nblk < base + L ? nblk : base + L;
 
     // one probe per distinct key in the warp
     u32 id = NO_ID;
@@ -202,7 +206,7 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
 
   if (valid) {
     for (int j = m + sl; j < max_blocks; j += L) ids_out[r * max_blocks + j] = -1;
-    if (sl == 0) matched[r] = m;
+    if (sl == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; }
   }
   // counters: warp sums, then fire-and-forget adds into one of LOOKUP_STRIPES stripes (no block barrier)
   u32 qb = (valid && sl == 0) ? (u32)nblk : 0, mb = (valid && sl == 0) ? (u32)m : 0;
@@ -254,9 +258,11 @@ __global__ void __launch_bounds__(128) chain_kernel(Store st, const u64* content
   for (int j = nblk + lane; j < max_blocks; j += 32) keys_out[r * max_blocks + j] = 0;
 }
 
-__global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* __restrict__ content, const long long* __restrict__ offsets,
+// `content` holds the content hashes on entry; the chained keys of every chunk that is probed are written over them
+// and hashed[r] says how many leading blocks of request r hold a key afterwards (kept for an insert of the same batch)
+__global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, u64* content, const long long* __restrict__ offsets,
                                                            int R, int max_blocks, u32 flags, u64 epoch, int* __restrict__ matched,
-                                                           int* __restrict__ ids_out, FetchLink fl) {
+                                                           int* __restrict__ ids_out, FetchLink fl, u32* __restrict__ hashed) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long r = warp;
@@ -265,8 +271,8 @@ __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* 
   u32 cnt0 = 0, cnt1 = 0;
   const int nblk = full_blocks(offsets, (int)r, st.block_tokens, max_blocks);
   const u64 inflation = st.policy ? st.ctrl->inflation : 0;
-  const u64* crow = content + r * max_blocks;
-  int m = 0;
+  u64* crow = content + r * max_blocks;
+  int m = 0, n_hashed = 0;
   u32 probes = 0, visited_sum = 0;
   u64 parent = st.root_key;
   u64 key = 0;
@@ -289,6 +295,8 @@ __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* 
       const int left = nblk - base - 32;
       next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
     }
+    if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
+    n_hashed = nblk < base + 32 ? nblk : base + 32;
     u32 id = NO_ID;
     if (active) {
       u32 visited;
@@ -323,7 +331,7 @@ __global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, const u64* 
   }
   if (fl.bt) link_count(st, cnt0, cnt1, lane);
   for (int j = m + lane; j < max_blocks; j += 32) ids_out[r * max_blocks + j] = -1;
-  if (lane == 0) matched[r] = m;
+  if (lane == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; }
   u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
   probes = __reduce_add_sync(FULL, probes);
   visited_sum = __reduce_add_sync(FULL, visited_sum);

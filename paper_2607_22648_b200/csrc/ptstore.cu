@@ -109,6 +109,9 @@ struct ptstore {
   u32 fetch_seq;         // sequence number of the last fetch call (tags the list heads; never 0)
   u32 coop_seq;          // cooperative launches so far (selects the barrier counter)
   u32 wait_limit;        // polls per bounded wait in the copy kernels' main loop
+  // the batch whose chained keys the last lookup left in `keys` / `prefix` (for ptstore_insert_after_lookup)
+  const void* lk_tokens; const void* lk_offsets; int lk_R, lk_max_blocks; bool lk_valid;
+  u64 inserts_resumed;   // inserts that resumed hashing behind a lookup's keys
   cudaEvent_t time_before, time_after;   // one-shot: recorded around the next HBM copy kernel (ptstore_time_next_copy)
   int coop_grid;         // CTAs a cooperative kernel may use: one per SM, at most MAX_COOP_GRID
   u64 epoch;
@@ -183,7 +186,7 @@ int launch_lookup(ptstore* h, const int* tokens, const long long* offsets, int R
                   int* ids, const FetchLink& fl, cudaStream_t s) {
   const long long warps = ((long long)R + (32 / L) - 1) / (32 / L);
   const int grid = (int)((warps * 32 + 255) / 256);
-  lookup_kernel<L><<<grid, 256, 0, s>>>(h->st, tokens, offsets, R, max_blocks, flags, h->epoch, matched, ids, fl);
+  lookup_kernel<L><<<grid, 256, 0, s>>>(h->st, tokens, offsets, R, max_blocks, flags, h->epoch, matched, ids, fl, h->keys, h->prefix);
   PTS_CHECK_LAUNCH(h);
   return PTSTORE_OK;
 }
@@ -435,13 +438,14 @@ int launch_fetch_copies(ptstore* h, const ptstore_paged_cache_t* dst, u32 seq, c
 int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks, uint32_t flags,
                 int32_t* matched_blocks, int32_t* block_ids, const FetchLink& fl, cudaStream_t s) {
   const long long* off = reinterpret_cast<const long long*>(offsets);
+  h->lk_tokens = tokens; h->lk_offsets = offsets; h->lk_R = R; h->lk_max_blocks = max_blocks; h->lk_valid = true;
   if (split_path(h, R, max_blocks)) {
     int rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
     if (rc) return rc;
     // few long requests: the chain loop of a warp is one long dependent sequence, so the lists are linked by a kernel of
     // its own with one thread per entry rather than inside that loop (13 us against 4 us for one 260-block prompt)
     FetchLink none = {};
-    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, none);
+    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, none, h->prefix);
     PTS_CHECK_LAUNCH(h);
     if (!fl.bt) return PTSTORE_OK;
     fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, block_ids, matched_blocks, R, max_blocks, fl);
@@ -627,9 +631,9 @@ int ptstore_fetch(ptstore_t* h, const int32_t* block_ids, const int32_t* matched
   return launch_fetch_copies(h, dst, fl.seq, s);
 }
 
-int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
-                   const ptstore_paged_cache_t* src, const int32_t* block_tables, int32_t* block_ids, int32_t* new_blocks,
-                   ptstore_stream_t stream) {
+static int insert_entry(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                        const ptstore_paged_cache_t* src, const int32_t* block_tables, int32_t* block_ids, int32_t* new_blocks,
+                        ptstore_stream_t stream, bool after_lookup) {
   int rc = check_batch(h, R, max_blocks);
   if (rc) return rc;
   if (R > 0 && (!offsets || !block_ids || !new_blocks)) return PTSTORE_E_INVAL;
@@ -651,6 +655,13 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   a.R = R; a.max_blocks = max_blocks;
   a.split = split_path(h, R, max_blocks) ? 1 : 0;
   a.keys = h->keys; a.eslot = h->eslot; a.cta_sums = h->cta_sums;
+  const int lanes = a.split ? 32 : lanes_for(h, R, max_blocks);
+  // the keys of this very batch, left by the last lookup: with a warp per request the chain resumes behind them
+  const bool resume = after_lookup && h->lk_valid && lanes == 32 && h->lk_tokens == tokens && h->lk_offsets == offsets && h->lk_R == R &&
+                      h->lk_max_blocks == max_blocks;
+  a.hashed = resume ? h->prefix : nullptr;
+  h->lk_valid = false;                        // this call overwrites the key scratch
+  if (resume) h->inserts_resumed += 1;
   a.bt = copy ? block_tables : nullptr;
   a.cache_blocks = copy ? src->num_blocks : 0;
   a.epoch = h->epoch;
@@ -658,7 +669,6 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   a.ids_out = block_ids; a.new_blocks = new_blocks;
   a.stash = h->stash;
   a.rebuild_threshold = rebuild_threshold(h);
-  const int lanes = a.split ? 32 : lanes_for(h, R, max_blocks);
   // CTAs: enough for one element per thread and for one sub-warp per request, at most one per SM
   const long long by_elems = (total + INS_THREADS - 1) / INS_THREADS;
   const long long by_reqs = ((long long)R * lanes + INS_THREADS - 1) / INS_THREADS;
@@ -674,6 +684,20 @@ int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, 
   if (copy) return launch_copy<COPY_INSERT>(h, to_paged(src), false, s, h->desc, &h->st.ctrl->n_pairs);
   return PTSTORE_OK;
 }
+
+int ptstore_insert(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                   const ptstore_paged_cache_t* src, const int32_t* block_tables, int32_t* block_ids, int32_t* new_blocks,
+                   ptstore_stream_t stream) {
+  return insert_entry(h, tokens, offsets, R, max_blocks, src, block_tables, block_ids, new_blocks, stream, false);
+}
+
+int ptstore_insert_after_lookup(ptstore_t* h, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
+                                const ptstore_paged_cache_t* src, const int32_t* block_tables, int32_t* block_ids, int32_t* new_blocks,
+                                ptstore_stream_t stream) {
+  return insert_entry(h, tokens, offsets, R, max_blocks, src, block_tables, block_ids, new_blocks, stream, true);
+}
+
+uint64_t ptstore_resumed_inserts(const ptstore_t* h) { return h ? h->inserts_resumed : 0; }
 
 int ptstore_release(ptstore_t* h, const int32_t* block_ids, const int32_t* matched_blocks, int32_t R, int32_t max_blocks,
                     ptstore_stream_t stream) {

@@ -49,7 +49,8 @@ class Pair:
     def lookup(self, seqs, max_blocks, flags=0):
         toks, offs = W.ragged(seqs)
         mo, io = self.o.lookup(toks, offs, max_blocks, flags)
-        mg, ig = self.g.lookup(dev(toks), dev(offs), max_blocks, flags)
+        self._last_batch = (dev(toks), dev(offs))
+        mg, ig = self.g.lookup(self._last_batch[0], self._last_batch[1], max_blocks, flags)
         assert (mo == mg.cpu().numpy()).all(), "matched lengths differ"
         assert (io == ig.cpu().numpy()).all(), "block ids differ"
         return mo, io, mg, ig
@@ -60,7 +61,8 @@ class Pair:
         gc = self.gpu_cache(np_cache)
         mo, io = self.o.lookup(toks, offs, max_blocks, flags)
         self.o.fetch(io, mo, np_cache, block_tables)
-        mg, ig = self.g.lookup_fetch(dev(toks), dev(offs), max_blocks, gc, dev(block_tables), flags)
+        self._last_batch = (dev(toks), dev(offs))          # kept: an insert_after_lookup must be handed these very tensors
+        mg, ig = self.g.lookup_fetch(self._last_batch[0], self._last_batch[1], max_blocks, gc, dev(block_tables), flags)
         assert (mo == mg.cpu().numpy()).all(), "matched lengths differ"
         assert (io == ig.cpu().numpy()).all(), "block ids differ"
         for l in range(self.shape.layers):
@@ -91,11 +93,13 @@ class Pair:
             assert torch.equal(gc.tensors[l].cpu(), torch.from_numpy(np_cache[l])), "fetched bytes differ in layer %d" % l
         return gc
 
-    def insert(self, seqs, max_blocks, np_cache=None, block_tables=None, tags=None):
+    def insert(self, seqs, max_blocks, np_cache=None, block_tables=None, tags=None, after_lookup=False):
+        """after_lookup: ptstore_insert_after_lookup with the device tensors of the preceding lookup / lookup_fetch."""
         toks, offs = W.ragged(seqs)
         io, no = self.o.insert(toks, offs, max_blocks, np_cache, block_tables, tags)
         gc = self.gpu_cache(np_cache) if np_cache is not None else None
-        ig, ng = self.g.insert(dev(toks), dev(offs), max_blocks, gc, dev(block_tables) if block_tables is not None else None)
+        dt, do = self._last_batch if after_lookup else (dev(toks), dev(offs))
+        ig, ng = self.g.insert(dt, do, max_blocks, gc, dev(block_tables) if block_tables is not None else None, after_lookup=after_lookup)
         assert (io == ig.cpu().numpy()).all(), "inserted ids differ"
         assert (no == ng.cpu().numpy()).all(), "new block counts differ"
         return io, no

@@ -707,7 +707,7 @@ def test_fused_step_lockstep(host, policy):
             asyn = bool(host) and step % 3 == 0
             p.reserve(sum(upper), mo, literal=bool(step % 2), asynchronous=asyn, max_victims=40 if step % 5 else 3,
                       headroom=(0, 0, 5)[step % 3])
-            p.insert(batch, mb, dst, bt)
+            p.insert(batch, mb, dst, bt, after_lookup=bool(step % 4))
             p.release(io, mo)
             p.check_status()
             if step % 10 == 9:
@@ -715,6 +715,38 @@ def test_fused_step_lockstep(host, policy):
                 p.check_counts()
         p.check_pools()
         p.check_counts()
+        p.close()
+
+
+def test_insert_after_lookup_resumes_behind_the_lookups_keys():
+    """Long prompts (a warp per request, with and without the separate content pass): the insert that follows a lookup of
+    the same device tensors reuses its keys; first-miss positions at the start, in the middle of a chunk, on a chunk border
+    and past the end are all covered, as is an eviction between the two calls and a fallback when the tensors differ."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    rng = np.random.default_rng(8)
+    for mb in (24, 100):                                   # 24: one chunk of 32 lanes per request; 100: the split path
+        p = Pair(sh, 600, max_requests=8, max_batch_blocks=8 * mb, byte_mode=False)
+        base = rng.integers(0, 50000, size=mb, dtype=np.int32)
+        p.insert([base[:70]], mb)                          # stored prefix of 70 (or 24) blocks
+        fresh = lambda n: rng.integers(50000, 99999, size=n, dtype=np.int32)
+        batch = [np.concatenate([base[:k], fresh(max(mb - k, 0))])[:mb] for k in (0, 5, 32, 64, 70)] + [base, base[:33], fresh(3)]
+        mo, io, _, _ = p.lookup(batch, mb, flags=1)
+        assert mo.tolist() == [min(k, mb, 70) for k in (0, 5, 32, 64, 70)] + [min(mb, 70), min(33, mb), 0]
+        p.evict(0, 3)                                      # keys stay valid across changes to the store
+        before = p.g.resumed_inserts()
+        p.insert(batch, mb, after_lookup=True)
+        assert p.g.resumed_inserts() == before + 1
+        p.release(io, mo)
+        p.lookup(batch, mb)
+        # other tensors than the lookup saw, or a call in between that used the key scratch: a plain insert
+        other = [fresh(mb) for _ in range(3)]
+        p.lookup(batch[:3], mb)
+        p.insert(other, mb, after_lookup=False)
+        p.insert(batch[:3], mb, after_lookup=True)
+        assert p.g.resumed_inserts() == before + 1
+        p.check_counts()
+        assert p.check_status() in (0, G.S_NOSPACE)
         p.close()
 
 
@@ -782,3 +814,35 @@ def test_bounded_wait_runs_out_and_the_store_stays_usable(engine):
     assert p.check_status() == 0
     p.check_counts()
     p.close()
+
+
+def test_copy_probe_moves_what_it_says():
+    """The measurement kernel really copies: a linear 1:1 copy reproduces the source, the mix writes every piece to two or
+    three destinations, the paged-like layout is a permutation of the pieces, and nothing else is touched."""
+    Pair, dev, G = _imports()
+    n, SB = 64 << 20, 32768
+    pieces = n // SB
+    src = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda")
+    dst = torch.full((3 * n,), 0xAB, dtype=torch.uint8, device="cuda")
+    status = G.copy_probe(src, dst, n, G.PROBE_COPY, scatter=False)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(dst[:n], src) and bool((dst[n:] == 0xAB).all())
+    dst.fill_(0xAB)
+    G.copy_probe(src, dst, n, G.PROBE_MIX, writes_x100=250, scatter=False, status=status)
+    torch.cuda.synchronize()
+    assert torch.equal(dst[:n], src) and torch.equal(dst[n:2 * n], src)
+    third = dst[2 * n:].view(pieces, SB)
+    written = (third != 0xAB).any(dim=1)
+    assert 0.4 < float(written.float().mean()) < 0.6
+    assert torch.equal(third[written], src.view(pieces, SB)[written])
+    dst.fill_(0xAB)
+    G.copy_probe(src, dst, n, G.PROBE_COPY, scatter=True, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(torch.sort(dst[:n].view(pieces, SB).long().sum(dim=1)).values, torch.sort(src.view(pieces, SB).long().sum(dim=1)).values)
+    before = dst.clone()
+    G.copy_probe(src, dst, n, G.PROBE_READ, status=status)
+    torch.cuda.synchronize()
+    assert torch.equal(dst, before) and int(status.item()) == 0
+    with pytest.raises(G.PTStoreError):
+        G.copy_probe(src, dst, n + 16, G.PROBE_COPY)
