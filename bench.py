@@ -418,7 +418,8 @@ def run_gpu(args):
     peak, peak_kind = measured_peak()
     host_tier_fetch = bool(wl.host_blocks) or args.engine == "vector"
     # the fetch copy kernel alone: bytes DRAM must move for it / its own duration
-    kern_ms = ev_ms["fetch_copy"] if ev_ms["fetch_copy"] > 0 else fetch_ms
+    # (with a host tier the fetch is two kernels, one per source tier: the call is timed instead)
+    kern_ms = ev_ms["fetch_copy"] if ev_ms["fetch_copy"] > 0 and not wl.host_blocks else fetch_ms
     fetch_dram = (main["distinct"] + main["fetched"]) * wl.sh.block_bytes
     ach = fetch_dram / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
     ach_delivered = main["fetched"] * block_rw / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
