@@ -43,7 +43,7 @@ NCU_READ_FACTOR = 1.00    # dram__bytes_read.sum / (distinct source blocks x blo
 NCU_WRITE_FACTOR = 0.99   # dram__bytes_write.sum / (delivered blocks x block bytes)
 FALLBACK_HBM_GBS = 6650.0
 # L2 read sectors per issued probe of lookup_kernel on the 10^6-node stress, from the ncu capture in profiles/
-L2_SECTORS_PER_PROBE = 9.4
+L2_SECTORS_PER_PROBE = 9.3
 
 
 def measured_peak():
@@ -434,7 +434,7 @@ def run_gpu(args):
                    "fill_steps": n_fill, "replicas": world},
         "value_kind": "bytes DRAM must move (distinct source blocks read once + delivered blocks written + 2 x stored blocks) / step time",
         "frac_of_nominal_8TBps": round(value / world / NOMINAL_HBM_GBS, 4),
-        # the same steps by the survey's convention: 2 x block bytes per delivered or stored block
+        # the same steps counting 2 x block bytes per delivered or stored block (one read and one write each)
         "value_delivered_bytes": round(delivered_all / (ms * 1e-3) / 1e9, 1),
         "per_step": {"blocks_fetched": main["fetched"] / K, "blocks_fetched_distinct": main["distinct"] / K, "blocks_inserted": main["inserted"] / K,
                      "blocks_dropped": main["dropped"] / K,
@@ -465,7 +465,7 @@ def run_gpu(args):
                          (NCU_READ_FACTOR * main["distinct"] + NCU_WRITE_FACTOR * main["fetched"]) * wl.sh.block_bytes / K),
                      "traffic_kind": "modelled from the small-case ncu capture (profiles/): DRAM bytes per distinct block read and per block "
                                      "written there, times this launch's distinct source blocks and delivered blocks",
-                     # the survey's convention (2 x block bytes per delivered block); above the copy peak because shared sources are read once
+                     # counting 2 x block bytes per delivered block; above the copy peak because shared sources are read once
                      "achieved_delivered_bytes": round(ach_delivered, 1), "frac_delivered_bytes": round(ach_delivered / peak, 4)},
     }
     if e2e:
@@ -489,7 +489,13 @@ def run_gpu(args):
             torch.cuda.empty_cache()
         if not args.no_ceilings and args.workload == "llama8b":
             ratio = main["fetched"] / max(main["distinct"], 1)
-            out["copy_engine_ceilings"] = ceilings_record(torch, writes_x100=int(round(ratio * 100)))
+            ceil = ceilings_record(torch, writes_x100=int(round(ratio * 100)))
+            out["copy_engine_ceilings"] = ceil
+            mix = [v for k, v in ceil.items() if k.startswith("mix_")][0]
+            # the same fraction against what the copy ring itself reaches, live, for a 1:1 copy and for this launch's mix
+            out["roofline"]["engine_ceilings"] = {"copy_1to1": ceil["copy_1to1"], "mix_of_this_fetch": mix, "writes_per_read": round(ratio, 2),
+                                                  "frac_of_copy_1to1": round(ach / ceil["copy_1to1"], 4), "frac_of_mix": round(ach / mix, 4),
+                                                  "kind": "ptstore_copy_probe in this run (the bulk ring over plain buffers)"}
             torch.cuda.empty_cache()
         if not args.no_lookup and args.workload == "llama8b":
             out["lookup"] = lookup_record(args, torch, K=args.lookup_calls, W_=5)["summary"]

@@ -18,6 +18,9 @@
  *     takes no lock.
  *   - ptstore_create makes cfg->device the calling thread's current CUDA device and leaves it so; every later call on
  *     the handle must be made with that device current (the library does not switch devices per call).
+ *   - The LRU clock, the sequence numbers that tag a fetch's lists and the choice of barrier counter are host-side
+ *     counters of the handle, passed to the kernels by value when a call is enqueued.  A call captured into a CUDA graph
+ *     would replay stale values, so enqueue calls directly; do not replay them from a captured graph.
  *   - Return value: PTSTORE_OK (0) or a negative PTSTORE_E_* code for conditions the host can see
  *     (bad arguments, CUDA launch errors).  Conditions only the device can see (pool exhausted,
  *     table full, block-table entry out of range, refcount underflow) are OR-ed as PTSTORE_S_* bits

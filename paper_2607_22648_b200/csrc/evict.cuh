@@ -113,9 +113,16 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
   const u32 tomb0 = c->tombstones;
   const u32 host_dropped = c->ev_host_dropped;
   u32 n = a.n;
-  if (a.want_free >= 0) {                      // reserve form: every thread sums the (short) list itself
-    long long need = a.want_free;
-    for (int i = 0; i < a.n_minus; ++i) { int m = a.minus[i]; need -= m > 0 ? m : 0; }
+  if (a.want_free >= 0) {                      // reserve form: every CTA sums the list for itself
+    u64 part = 0;
+    for (int i = threadIdx.x; i < a.n_minus; i += EV_THREADS) { const int m = a.minus[i]; part += m > 0 ? (u64)m : 0; }
+    for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(FULL, part, o);
+    if (lane == 0) red[w][0] = part;
+    __syncthreads();
+    part = 0;
+    for (int i = 0; i < EV_WARPS; ++i) part += red[i][0];
+    __syncthreads();                             // red is used again below
+    long long need = a.want_free - (long long)part;
     need -= (long long)count0;
     if (need > 0) need += (long long)a.n;                 // short of room: evict `n` blocks more than needed right now
     n = need > 0 ? (need > 0x7FFFFFFFll ? 0x7FFFFFFFu : (u32)need) : 0u;
