@@ -85,3 +85,33 @@ int main(void) {
         got = [int(x) for x in subprocess.check_output([exe]).split()]
     want = [C.sizeof(Config), Config.salt.offset, Config.table_slots.offset, Config.device.offset, C.sizeof(PagedCache), C.sizeof(Stats)]
     assert got == want
+
+
+def test_new_entry_points_refuse_bad_arguments_on_the_host():
+    """Argument checks that need no device: a null handle, null buffers, sizes out of range."""
+    lib = C.CDLL(build.build())
+    vp, i32, u32, u64, i64 = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64, C.c_int64
+    lib.ptstore_reserve.argtypes = [vp, i64, i32, vp, i32, u32, vp, vp, i32, vp]
+    lib.ptstore_lookup_fetch.argtypes = [vp, vp, vp, i32, i32, u32, vp, vp, vp, vp, vp]
+    lib.ptstore_insert_after_lookup.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.ptstore_set_wait_limit.argtypes = [vp, u32]
+    lib.ptstore_time_next_copy.argtypes = [vp, vp, vp]
+    lib.ptstore_copy_probe.argtypes = [vp, vp, u64, i32, u32, i32, u32, i32, i32, vp, vp]
+    lib.ptstore_resumed_inserts.restype = u64
+    lib.ptstore_resumed_inserts.argtypes = [vp]
+    E_INVAL = -1
+    assert lib.ptstore_reserve(None, 10, 0, None, 0, 0, None, None, 0, None) == E_INVAL
+    assert lib.ptstore_lookup_fetch(None, None, None, 1, 1, 0, None, None, None, None, None) == E_INVAL
+    assert lib.ptstore_insert_after_lookup(None, None, None, 1, 1, None, None, None, None, None) == E_INVAL
+    assert lib.ptstore_set_wait_limit(None, 1) == E_INVAL
+    assert lib.ptstore_time_next_copy(None, None, None) == E_INVAL
+    assert lib.ptstore_resumed_inserts(None) == 0
+    # the copy probe checks pointers, alignment, mode, ring geometry and sizes before it touches the device
+    a = 1 << 20
+    assert lib.ptstore_copy_probe(None, a, 1 << 26, 2, 100, 3, 32768, 1, 0, a, None) == E_INVAL
+    assert lib.ptstore_copy_probe(a, a + 8, 1 << 26, 2, 100, 3, 32768, 1, 0, a, None) == E_INVAL          # misaligned
+    assert lib.ptstore_copy_probe(a, a, 1 << 26, 7, 100, 3, 32768, 1, 0, a, None) == E_INVAL              # unknown mode
+    assert lib.ptstore_copy_probe(a, a, 1 << 26, 2, 100, 1, 32768, 1, 0, a, None) == E_INVAL              # one stage is no ring
+    assert lib.ptstore_copy_probe(a, a, 1 << 26, 2, 100, 8, 32768, 1, 0, a, None) == E_INVAL              # ring above 200 KiB
+    assert lib.ptstore_copy_probe(a, a, 1 << 26, 3, 50, 3, 32768, 1, 0, a, None) == E_INVAL               # fewer than one store per load
+    assert lib.ptstore_copy_probe(a, a, (1 << 26) + 32768, 2, 100, 3, 32768, 1, 0, a, None) == E_INVAL    # not a whole number of units
