@@ -1,7 +1,8 @@
 // CPU oracle of the prefix tensor store — TEST INFRASTRUCTURE, not a product path.
 //
-// A plain, single-threaded restatement of what the prefix-hit path computes, used only by the tests,
-// the smoke check and the CPU-baseline leg of the benchmark.  It shares no code with the CUDA
+// A plain restatement of what the prefix-hit path computes, used only by the tests, the smoke check and
+// the CPU-baseline leg of the benchmark.  Single-threaded, except for one function that splits the two
+// read-only phases over host threads for the all-cores baseline (oracle_lookup_fetch_threads).  It shares no code with the CUDA
 // library and never calls it.  Nodes are found by comparing TOKENS (a pointer trie whose children are
 // keyed by the token content of a block), never by hash, so that a key collision in the hashed GPU
 // table would show up as a disagreement rather than be reproduced.

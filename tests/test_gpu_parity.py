@@ -389,6 +389,14 @@ def test_edge_cases_and_errors():
     assert e.value.code == G.E_INVAL
     with pytest.raises(G.PTStoreError):
         g.evict(1, 1)                                    # no host tier
+    with pytest.raises(G.PTStoreError) as e:
+        g.reserve(4, torch.zeros(5, dtype=torch.int32, device="cuda"))       # more entries than max_requests
+    assert e.value.code == G.E_LIMIT
+    with pytest.raises(G.PTStoreError) as e:
+        g.reserve(-1)
+    assert e.value.code == G.E_INVAL
+    ne, _ = g.reserve(3)                                 # an empty store has room: nothing to evict, no victim list wanted
+    assert ne.tolist() == [0, 0]
     # out-of-range block table entries and ids are skipped and flagged, nothing else is touched
     s = np.arange(16, dtype=np.int32)
     src = W.random_kv_cache(0, sh, 4)
