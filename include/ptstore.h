@@ -205,7 +205,7 @@ int ptstore_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets,
  * application is the latency of the pair).  Same results as the two calls: matched_blocks and block_ids are written
  * as by ptstore_lookup(flags), and every matched block j of request r is copied to cache block
  * block_tables[r*max_blocks+j] as by ptstore_fetch.  The lookup kernel builds the copy lists itself while it probes,
- * so the pair costs two kernel launches (three when requests are few and long, three or four with a host tier).
+ * so the pair costs two kernel launches (three with a host tier).
  */
 int ptstore_lookup_fetch(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
                          uint32_t flags, const ptstore_paged_cache_t* dst /*host struct*/,

@@ -224,9 +224,9 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
 // With a whole warp per request the fused kernel above is one dependent chain per 32-block chunk: token loads ->
 // content hashes -> 32 chain steps -> probe.  For long prompts (hundreds of blocks, a handful of requests) that
 // serial latency is all there is.  Here the content hashes of ALL blocks are computed first by one thread per block
-// (content_kernel), and the per-request warp only chains and probes; the probe loads of a chunk are in flight while
-// the keys of the next chunk are chained (the chain does not depend on the probe result; if the chunk then turns out
-// to hold the first miss the extra chain is discarded).
+// (content_kernel for ptstore_hash, the first phase of lookup_long_kernel for lookups), and the per-request warp only
+// chains and probes; the probe loads of a chunk are in flight while the keys of the next chunk are chained (the chain
+// does not depend on the probe result; if the chunk then turns out to hold the first miss the extra chain is discarded).
 __global__ void __launch_bounds__(256) content_kernel(Store st, const int* __restrict__ tokens, const long long* __restrict__ offsets,
                                                       int R, int max_blocks, u64* __restrict__ content_out) {
   const long long total = (long long)R * max_blocks;
@@ -258,88 +258,109 @@ __global__ void __launch_bounds__(128) chain_kernel(Store st, const u64* content
   for (int j = nblk + lane; j < max_blocks; j += 32) keys_out[r * max_blocks + j] = 0;
 }
 
-// `content` holds the content hashes on entry; the chained keys of every chunk that is probed are written over them
-// and hashed[r] says how many leading blocks of request r hold a key afterwards (kept for an insert of the same batch)
-__global__ void __launch_bounds__(128) lookup_chain_kernel(Store st, u64* content, const long long* __restrict__ offsets,
-                                                           int R, int max_blocks, u32 flags, u64 epoch, int* __restrict__ matched,
-                                                           int* __restrict__ ids_out, FetchLink fl, u32* __restrict__ hashed) {
+// One CTA per request, three phases in one launch.
+//   1. all threads: content hashes of the request's blocks into `scratch` (one thread per block);
+//   2. warp 0: the chain, the probes and the first miss, as described above; the chained keys of every chunk that is
+//      probed are written over the content hashes and hashed[r] says how many leading blocks of request r hold a key
+//      afterwards (kept for an insert of the same batch);
+//   3. all threads: the -1 padding of the ids and, with a fetch attached, the linking of the matched blocks to their
+//      source blocks (one thread per entry: inside the chain loop the same work cost three dependent memory round
+//      trips per chunk of a serial loop).
+constexpr int LONG_THREADS = 256;
+__global__ void __launch_bounds__(LONG_THREADS) lookup_long_kernel(Store st, const int* __restrict__ tokens, u64* scratch,
+                                                                  const long long* __restrict__ offsets, int R, int max_blocks,
+                                                                  u32 flags, u64 epoch, int* __restrict__ matched,
+                                                                  int* __restrict__ ids_out, FetchLink fl, u32* __restrict__ hashed) {
+  __shared__ int s_m;
   const int lane = threadIdx.x & 31;
-  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long r = warp;
+  const long long r = blockIdx.x;
   if (fl.bt && blockIdx.x == 0 && threadIdx.x == 0) link_prepare_next(st, fl);
-  if (r >= R) return;
-  u32 cnt0 = 0, cnt1 = 0;
   const int nblk = full_blocks(offsets, (int)r, st.block_tokens, max_blocks);
-  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
-  u64* crow = content + r * max_blocks;
-  int m = 0, n_hashed = 0;
-  u32 probes = 0, visited_sum = 0;
-  u64 parent = st.root_key;
-  u64 key = 0;
-  u64 c_next = 0;                                  // content hashes of the chunk after the current one, loaded a chunk ahead
-  if (nblk > 0) {
-    const u64 c0 = lane < nblk ? crow[lane] : 0;
-    c_next = 32 + lane < nblk ? crow[32 + lane] : 0;
-    key = chain_chunk<32>(parent, c0, lane, nblk < 32 ? nblk : 32);
+  u64* crow = scratch + r * max_blocks;
+  {
+    const int* t0 = tokens + offsets[r];
+    for (int j = threadIdx.x; j < nblk; j += LONG_THREADS) crow[j] = content_block(t0 + (long long)j * st.block_tokens, st.block_tokens);
   }
-  for (int base = 0; base < nblk; base += 32) {
-    const int j = base + lane;
-    const bool active = j < nblk;
-    ProbeWindow w;
-    if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
-    u64 next_key = 0;
-    if (base + 32 < nblk) {                                       // ... while the next chunk is chained
-      const u64 cn = c_next;
-      c_next = base + 64 + lane < nblk ? crow[base + 64 + lane] : 0;
-      u64 p = __shfl_sync(FULL, key, 31);
-      const int left = nblk - base - 32;
-      next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const u64 inflation = st.policy ? st.ctrl->inflation : 0;
+    int m = 0, n_hashed = 0;
+    u32 probes = 0, visited_sum = 0;
+    u64 parent = st.root_key;
+    u64 key = 0;
+    u64 c_next = 0;                                  // content hashes of the chunk after the current one, loaded a chunk ahead
+    if (nblk > 0) {
+      const u64 c0 = lane < nblk ? crow[lane] : 0;
+      c_next = 32 + lane < nblk ? crow[32 + lane] : 0;
+      key = chain_chunk<32>(parent, c0, lane, nblk < 32 ? nblk : 32);
     }
-    if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
-    n_hashed = nblk < base + 32 ? nblk : base + 32;
-    u32 id = NO_ID;
-    if (active) {
-      u32 visited;
-      id = probe_finish(st.table, st.slots, key, w, &visited);
-      probes += 1;
-      visited_sum += visited;
-    }
-    const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
-    const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);
-    const bool hit = active && lane < nf;
-    const unsigned hm = __ballot_sync(FULL, hit);
-    if (hit) {
-      ids_out[r * max_blocks + j] = (int)id;
-      const bool touch = !(flags & F_NO_TOUCH);
-      if (touch && st.policy == 0) st.m_last[id] = epoch;
-      if ((flags & F_PIN) || (touch && st.policy)) {
-        const unsigned same = __match_any_sync(hm, id);            // ids of one request are distinct: groups of one
-        if (lane == __ffs(same) - 1) {
-          const u32 cnt = (u32)__popc(same);
-          if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
-          if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
+    for (int base = 0; base < nblk; base += 32) {
+      const int j = base + lane;
+      const bool active = j < nblk;
+      ProbeWindow w;
+      if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
+      u64 next_key = 0;
+      if (base + 32 < nblk) {                                       // ... while the next chunk is chained
+        const u64 cn = c_next;
+        c_next = base + 64 + lane < nblk ? crow[base + 64 + lane] : 0;
+        u64 p = __shfl_sync(FULL, key, 31);
+        const int left = nblk - base - 32;
+        next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
+      }
+      if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
+      n_hashed = nblk < base + 32 ? nblk : base + 32;
+      u32 id = NO_ID;
+      if (active) {
+        u32 visited;
+        id = probe_finish(st.table, st.slots, key, w, &visited);
+        probes += 1;
+        visited_sum += visited;
+      }
+      const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
+      const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);
+      const bool hit = active && lane < nf;
+      const unsigned hm = __ballot_sync(FULL, hit);
+      if (hit) {
+        ids_out[r * max_blocks + j] = (int)id;
+        const bool touch = !(flags & F_NO_TOUCH);
+        if (touch && st.policy == 0) st.m_last[id] = epoch;
+        if ((flags & F_PIN) || (touch && st.policy)) {
+          const unsigned same = __match_any_sync(hm, id);            // ids of one request are distinct: groups of one
+          if (lane == __ffs(same) - 1) {
+            const u32 cnt = (u32)__popc(same);
+            if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
+            if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
+          }
         }
       }
+      m += nf;
+      if (nf < 32) break;
+      key = next_key;
     }
-    if (fl.bt) {
-      const int opened = hit ? link_entry(st, fl, r * max_blocks + j, (int)id, cnt0, cnt1) : 0;
-      link_append(st, fl, opened, (int)id, lane);
+    if (lane == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; s_m = m; }
+    u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
+    probes = __reduce_add_sync(FULL, probes);
+    visited_sum = __reduce_add_sync(FULL, visited_sum);
+    qb = __reduce_add_sync(FULL, qb);
+    mb = __reduce_add_sync(FULL, mb);
+    if (lane < 4) {
+      const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
+      if (v) atomicAdd(&st.ctrl->lookup_stripes[r % LOOKUP_STRIPES][lane], (u64)v);
     }
-    m += nf;
-    if (nf < 32) break;
-    key = next_key;
   }
-  if (fl.bt) link_count(st, cnt0, cnt1, lane);
-  for (int j = m + lane; j < max_blocks; j += 32) ids_out[r * max_blocks + j] = -1;
-  if (lane == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; }
-  u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
-  probes = __reduce_add_sync(FULL, probes);
-  visited_sum = __reduce_add_sync(FULL, visited_sum);
-  qb = __reduce_add_sync(FULL, qb);
-  mb = __reduce_add_sync(FULL, mb);
-  if (lane < 4) {
-    const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
-    if (v) atomicAdd(&st.ctrl->lookup_stripes[warp % LOOKUP_STRIPES][lane], (u64)v);
+  __syncthreads();
+  const int m = s_m;
+  for (int j = m + threadIdx.x; j < max_blocks; j += LONG_THREADS) ids_out[r * max_blocks + j] = -1;
+  if (fl.bt) {
+    u32 cnt0 = 0, cnt1 = 0;
+    for (int j0 = 0; j0 < m; j0 += LONG_THREADS) {
+      const int j = j0 + threadIdx.x;
+      const bool hit = j < m;
+      const int id = hit ? ids_out[r * max_blocks + j] : -1;
+      const int opened = hit ? link_entry(st, fl, r * max_blocks + j, id, cnt0, cnt1) : 0;
+      link_append(st, fl, opened, id, lane);
+    }
+    link_count(st, cnt0, cnt1, lane);
   }
 }
 

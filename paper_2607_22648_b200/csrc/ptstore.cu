@@ -439,16 +439,9 @@ int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32
                 int32_t* matched_blocks, int32_t* block_ids, const FetchLink& fl, cudaStream_t s) {
   const long long* off = reinterpret_cast<const long long*>(offsets);
   h->lk_tokens = tokens; h->lk_offsets = offsets; h->lk_R = R; h->lk_max_blocks = max_blocks; h->lk_valid = true;
-  if (split_path(h, R, max_blocks)) {
-    int rc = launch_content(h, tokens, off, R, max_blocks, h->keys, s);
-    if (rc) return rc;
-    // few long requests: the chain loop of a warp is one long dependent sequence, so the lists are linked by a kernel of
-    // its own with one thread per entry rather than inside that loop (13 us against 4 us for one 260-block prompt)
-    FetchLink none = {};
-    lookup_chain_kernel<<<(R + 3) / 4, 128, 0, s>>>(h->st, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, none, h->prefix);
-    PTS_CHECK_LAUNCH(h);
-    if (!fl.bt) return PTSTORE_OK;
-    fetch_link_kernel<<<grid_for((long long)R * max_blocks, 256, h->sms * 8), 256, 0, s>>>(h->st, block_ids, matched_blocks, R, max_blocks, fl);
+  if (split_path(h, R, max_blocks)) {      // few long requests: one CTA per request does content hashes, chain and list linking
+    lookup_long_kernel<<<R, LONG_THREADS, 0, s>>>(h->st, tokens, h->keys, off, R, max_blocks, flags, h->epoch, matched_blocks, block_ids, fl,
+                                                  h->prefix);
     PTS_CHECK_LAUNCH(h);
     return PTSTORE_OK;
   }
