@@ -493,8 +493,14 @@ def run_gpu(args):
             out["copy_engine_ceilings"] = ceil
             mix = [v for k, v in ceil.items() if k.startswith("mix_")][0]
             # the same fraction against what the copy ring itself reaches, live, for a 1:1 copy and for this launch's mix
+            # loads and stores measured apart, combined for this launch's byte counts: time = read bytes / read ceiling + written
+            # bytes / write ceiling (the memory serves one direction at a time)
+            rd, wr = ceil["read_only_4_stages"], ceil["write_only"]
+            harmonic = (1 + ratio) / (1 / rd + ratio / wr)
             out["roofline"]["engine_ceilings"] = {"copy_1to1": ceil["copy_1to1"], "mix_of_this_fetch": mix, "writes_per_read": round(ratio, 2),
+                                                  "reads_alone": rd, "writes_alone": wr, "reads_and_writes_in_turn": round(harmonic, 1),
                                                   "frac_of_copy_1to1": round(ach / ceil["copy_1to1"], 4), "frac_of_mix": round(ach / mix, 4),
+                                                  "frac_of_reads_and_writes_in_turn": round(ach / harmonic, 4),
                                                   "kind": "ptstore_copy_probe in this run (the bulk ring over plain buffers)"}
             torch.cuda.empty_cache()
         if not args.no_lookup and args.workload == "llama8b":
