@@ -171,3 +171,37 @@ def test_large_blocks_of_1024_tokens():
     assert matched > 20 and srv.sampled_chunks >= 256
     print("1024-token blocks: chunk %d KiB, block %d MiB, matched %d blocks" % (sh.chunk_bytes >> 10, sh.block_bytes >> 20, matched))
     srv.close()
+
+
+@pytest.mark.parametrize("host,policy,shape", [(0, "lru", "long16"), (4000, "gdsf", "long4"), (0, "gdsf", "short1500"), (20000, "lru", "short1100")])
+def test_medium_serving_loops_where_cooperative_kernels_span_several_ctas(host, policy, shape):
+    """Medium sizes between the small lock-step tests and the full-size ones: eviction over 3,000-15,000 block ids (6-30 CTAs
+    meeting at grid barriers), insert metadata over 2,500-20,000 elements (3-20 CTAs), long prompts (one CTA per request)
+    and thousands of short ones (sub-warps, lists linked inside the chunk loop); two thirds of the steps use the fused calls,
+    the rest the separate ones with promotion and asynchronous demotion; table rebuilds happen every few steps."""
+    from tests.serving import LockstepServing
+    if shape.startswith("long"):
+        bt = int(shape[4:])
+        sh = W.KVShape(2, 1, 8, bt)
+        st = W.doc_stream(900, sh, n_docs=80, len_range=(150, 1600), zipf_s=1.0, vocab=5000, suffix_range=(3, 70))
+        batch, hbm, steps, promote = (24 if bt == 16 else 12), (3000 if bt == 16 else 6000), 120, 40
+    else:
+        batch = int(shape[5:])
+        sh = W.KVShape(1, 1, 8, 16)
+        st = W.doc_stream(700, sh, n_docs=4000, len_range=(16, 128) if batch == 1500 else (100, 250), zipf_s=0.9, vocab=3000, suffix_range=(1, 40))
+        hbm, steps, promote = 15000, 40, 300
+    mb = st.max_blocks
+    srv = LockstepServing(sh, hbm, host, batch, mb, batch * mb + 8, seed=3, policy=policy)
+    evicting = 0
+    for k in range(steps):
+        seqs, tags = st.batch(batch)
+        fused = k % 3 != 2
+        r = srv.step(seqs, tags, sample=1, check_all=(k % 10 == 0), fused=fused, promote=(0 if fused or not host else promote),
+                     async_demote=(bool(host) and not fused and k % 2 == 0))
+        evicting += r["evicted"] is not None
+    s = srv.check_counts()
+    assert srv.check_pool(16) > 0
+    assert evicting > steps // 2 and s.rebuilds > 0
+    if shape.startswith("long"):
+        assert srv.g.resumed_inserts() == len([k for k in range(steps) if k % 3 != 2])
+    srv.close()
