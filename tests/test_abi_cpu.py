@@ -115,3 +115,23 @@ def test_new_entry_points_refuse_bad_arguments_on_the_host():
     assert lib.ptstore_copy_probe(a, a, 1 << 26, 2, 100, 8, 32768, 1, 0, a, None) == E_INVAL              # ring above 200 KiB
     assert lib.ptstore_copy_probe(a, a, 1 << 26, 3, 50, 3, 32768, 1, 0, a, None) == E_INVAL               # fewer than one store per load
     assert lib.ptstore_copy_probe(a, a, (1 << 26) + 32768, 2, 100, 3, 32768, 1, 0, a, None) == E_INVAL    # not a whole number of units
+
+
+def build_c_client(out_dir):
+    """Compile and link tests/abi_client.c (plain C99) against the library and the CUDA runtime; returns the executable."""
+    import subprocess
+    lib = build.build()
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    exe = os.path.join(out_dir, "abi_client")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-O1", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(cuda, "include"),
+                           os.path.join(ROOT, "tests", "abi_client.c"), "-o", exe, lib, "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                           "-Wl,-rpath," + os.path.dirname(lib), "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+    return exe
+
+
+def test_a_plain_c_program_compiles_and_links_against_the_library():
+    """The boundary is usable from C with nothing but the header, the shared library and the CUDA runtime (the program
+    itself runs in the GPU tests)."""
+    import tempfile
+    with tempfile.TemporaryDirectory() as d:
+        assert os.path.exists(build_c_client(d))

@@ -854,3 +854,16 @@ def test_copy_probe_moves_what_it_says():
     assert torch.equal(dst, before) and int(status.item()) == 0
     with pytest.raises(G.PTStoreError):
         G.copy_probe(src, dst, n + 16, G.PROBE_COPY)
+
+
+def test_plain_c_client_runs_the_path_through_the_c_abi():
+    """tests/abi_client.c: insert, fused lookup + gather, reserve, insert, release from a C program that links the library
+    directly; it checks ids, matched lengths, counters and every fetched byte itself."""
+    import subprocess
+    import tempfile
+    from tests.test_abi_cpu import build_c_client
+    with tempfile.TemporaryDirectory() as d:
+        exe = build_c_client(d)
+        r = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+        assert r.returncode == 0, r.stdout + r.stderr
+        assert r.stdout.startswith("abi client ok")
