@@ -40,25 +40,22 @@ struct Ctrl {
   u32 status;
   u32 pad0;
   // per-call scalars produced by one kernel and consumed by the next
-  u32 n_pairs;          // fetch / insert / promote: entries in the copy descriptor list
-  u32 n_pairs_host;     // fetch: distinct host-tier source blocks (their descriptors form a list of their own)
+  u32 n_pairs;          // insert / promote: entries in the copy descriptor list
   u32 n_pairs_tier;     // demotion: entries in its own descriptor list (its copy may run on the library's side stream)
   u32 ins_total_new;    // insert: new unique nodes presented
-  u32 ins_granted;      // insert: of those, how many got a block
-  u32 ins_base;         // insert: ring head before this call
-  u32 ev_want;          // evict: victims still wanted by the current phase
-  u32 ev_cand;          // evict: candidates collected
-  u32 ev_take;          // evict: victims taken by the current phase
+  u32 ins_granted;      // insert / promote: of those, how many got a block
+  u32 ins_base;         // insert / promote: ring head before this call
+  u32 ev_take;          // promote: where the freed host ids go in the host ring
   u32 ev_host_dropped;  // evict: host-tier drops that made room for a demotion
   u32 live[2];
   u32 tombstones;
-  u32 work_counter;     // spare
+  u32 pad1;
   // fetch: per-call scalars, double buffered by the call's sequence number so that no launch is needed to clear them:
   // call k uses entry k & 1 and zeroes entry (k + 1) & 1 for the call after it
   u32 f_pairs[2];       // distinct HBM-tier source blocks = entries of the descriptor list
   u32 f_pairs_host[2];  // distinct host-tier source blocks (a descriptor list of their own)
   u32 f_work[2];        // next work unit to hand out (dynamic dealing inside the copy kernel)
-  u32 pad1[2];
+  u32 pad2[2];
   // arrival counters of the grid-wide barriers of cooperative kernels: launch k uses entry k % BAR_SLOTS and zeroes
   // the entry half a ring ahead, so a counter is always zero when its turn comes, whatever happened to earlier launches
   u32 bar[64];
