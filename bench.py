@@ -634,9 +634,6 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
         wall = []
         for _ in range(iters):
             evs = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-            ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            ca.record(); cb.record()                                    # bring the events into existence
-            lib.ptstore_time_next_copy(h, ca.cuda_event, cb.cuda_event)  # the gather kernel of the lookup_fetch below
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             for q, (_n, f, a) in enumerate(calls(k)):
@@ -646,7 +643,6 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
             wall.append((time.perf_counter() - t0) * 1e6)
             for q, (n, _f, _a) in enumerate(calls(k)):
                 per_call.setdefault(n, []).append(evs[q].elapsed_time(evs[q + 1]) * 1e3)
-            per_call.setdefault("gather_kernel_of_lookup_fetch", []).append(ca.elapsed_time(cb) * 1e3)
             k += 1
         fetched = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) / iters
         inserted = (s1.blocks_inserted - s0.blocks_inserted) / iters
@@ -658,7 +654,8 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
                               "launches_per_step": (l1 - l0) / iters, "blocks_fetched": fetched, "blocks_inserted": inserted,
                               "blocks_evicted": dropped, "copy_bytes": copy_bytes, "copy_bound_us": round(bound_us, 1),
                               "step_over_copy_bound": round(step_us / bound_us, 3), "gbps": round(copy_bytes / step_us / 1e3, 1)}
-    assert st.status() == 0
+        status = st.status()
+        assert status == 0, "status word 0x%x after the batch-%d steps" % (status, b)
     res["config"] = {"kv_shape": "32L x 8H x 128 bf16, block 16", "prompt": "%d-token stored document + %d fresh tokens" % (doc_tokens, suffix_tokens),
                      "pool_blocks": pool, "docs": n_docs, "iters": iters, "reserve_headroom": headroom,
                      "copy_bound": "bytes of the step's fetch and insert copies (read + write) / measured copy bandwidth"}

@@ -379,10 +379,13 @@ __global__ void __launch_bounds__(256) store_init_kernel(Store st, u64* __restri
     else st.ring_ids[1][i - st.n[0]] = (int)i;
   }
 }
-__global__ void ctrl_init_kernel(Store st) {
+// `progress`: the per-request progress words of the fused lookup + gather.  They carry the launch number as a tag, launch
+// numbers start at 1, and the workspace may hold the words of an earlier handle: cleared here.
+__global__ void ctrl_init_kernel(Store st, u64* __restrict__ progress, int n_progress) {
   Ctrl* c = st.ctrl;
   unsigned char* p = reinterpret_cast<unsigned char*>(c);
   for (size_t i = 0; i < sizeof(Ctrl); ++i) p[i] = 0;
+  for (int i = 0; i < n_progress; ++i) progress[i] = 0;
   c->ring[0].count = st.n[0];
   c->ring[1].count = st.n[1];
 }

@@ -266,6 +266,95 @@ __global__ void __launch_bounds__(128) chain_kernel(Store st, const u64* content
 //   3. all threads: the -1 padding of the ids and, with a fetch attached, the linking of the matched blocks to their
 //      source blocks (one thread per entry: inside the chain loop the same work cost three dependent memory round
 //      trips per chunk of a serial loop).
+// Progress word of a request in the fused lookup + gather kernel: (launch tag << 32) | (done << 31) | blocks matched so far.
+// A word with another tag was written by an earlier launch and reads as "nothing yet".
+__device__ __forceinline__ void publish_progress(u64* progress, long long r, u32 tag, u32 count, bool done) {
+  const u64 v = ((u64)tag << 32) | (done ? 0x80000000ull : 0ull) | (u64)count;
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(progress + r), "l"(v) : "memory");
+}
+
+// One warp: chain, probes, first miss, pins and stamps of request r, whose content hashes are in crow.  The chained keys
+// of every chunk that is probed are written over the content hashes and hashed[r] says how many leading blocks hold a key
+// afterwards (kept for an insert of the same batch).  With `progress` the number of blocks matched so far is published after
+// every chunk, so that another CTA can start copying them.  Returns the matched length (in every lane).
+__device__ __forceinline__ int chain_probe_request(const Store& st, u64* crow, int nblk, long long r, int max_blocks, u32 flags, u64 epoch,
+                                                   int* __restrict__ matched, int* __restrict__ ids_out, u32* __restrict__ hashed,
+                                                   u64* progress, u32 tag, int lane) {
+  const u64 inflation = st.policy ? st.ctrl->inflation : 0;
+  int m = 0, n_hashed = 0;
+  u32 probes = 0, visited_sum = 0;
+  u64 parent = st.root_key;
+  u64 key = 0;
+  u64 c_next = 0;                                  // content hashes of the chunk after the current one, loaded a chunk ahead
+  if (nblk > 0) {
+    const u64 c0 = lane < nblk ? crow[lane] : 0;
+    c_next = 32 + lane < nblk ? crow[32 + lane] : 0;
+    key = chain_chunk<32>(parent, c0, lane, nblk < 32 ? nblk : 32);
+  }
+  for (int base = 0; base < nblk; base += 32) {
+    const int j = base + lane;
+    const bool active = j < nblk;
+    ProbeWindow w;
+    if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
+    u64 next_key = 0;
+    if (base + 32 < nblk) {                                       // ... while the next chunk is chained
+      const u64 cn = c_next;
+      c_next = base + 64 + lane < nblk ? crow[base + 64 + lane] : 0;
+      u64 p = __shfl_sync(FULL, key, 31);
+      const int left = nblk - base - 32;
+      next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
+    }
+    if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
+    n_hashed = nblk < base + 32 ? nblk : base + 32;
+    u32 id = NO_ID;
+    if (active) {
+      u32 visited;
+      id = probe_finish(st.table, st.slots, key, w, &visited);
+      probes += 1;
+      visited_sum += visited;
+    }
+    const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
+    const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);
+    const bool hit = active && lane < nf;
+    const unsigned hm = __ballot_sync(FULL, hit);
+    if (hit) {
+      ids_out[r * max_blocks + j] = (int)id;
+      const bool touch = !(flags & F_NO_TOUCH);
+      if (touch && st.policy == 0) st.m_last[id] = epoch;
+      if ((flags & F_PIN) || (touch && st.policy)) {
+        const unsigned same = __match_any_sync(hm, id);            // ids of one request are distinct: groups of one
+        if (lane == __ffs(same) - 1) {
+          const u32 cnt = (u32)__popc(same);
+          if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
+          if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
+        }
+      }
+    }
+    m += nf;
+    if (progress && nf == 32 && base + 32 < nblk) {              // more to come: let the copies of this chunk start
+      __syncwarp();
+      if (lane == 0) { __threadfence(); publish_progress(progress, r, tag, (u32)m, false); }
+    }
+    if (nf < 32) break;
+    key = next_key;
+  }
+  if (lane == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; }
+  if (progress) {
+    __syncwarp();
+    if (lane == 0) { __threadfence(); publish_progress(progress, r, tag, (u32)m, true); }
+  }
+  u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
+  probes = __reduce_add_sync(FULL, probes);
+  visited_sum = __reduce_add_sync(FULL, visited_sum);
+  qb = __reduce_add_sync(FULL, qb);
+  mb = __reduce_add_sync(FULL, mb);
+  if (lane < 4) {
+    const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
+    if (v) atomicAdd(&st.ctrl->lookup_stripes[r % LOOKUP_STRIPES][lane], (u64)v);
+  }
+  return m;
+}
+
 constexpr int LONG_THREADS = 256;
 __global__ void __launch_bounds__(LONG_THREADS) lookup_long_kernel(Store st, const int* __restrict__ tokens, u64* scratch,
                                                                   const long long* __restrict__ offsets, int R, int max_blocks,
@@ -283,70 +372,8 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_long_kernel(Store st, con
   }
   __syncthreads();
   if (threadIdx.x < 32) {
-    const u64 inflation = st.policy ? st.ctrl->inflation : 0;
-    int m = 0, n_hashed = 0;
-    u32 probes = 0, visited_sum = 0;
-    u64 parent = st.root_key;
-    u64 key = 0;
-    u64 c_next = 0;                                  // content hashes of the chunk after the current one, loaded a chunk ahead
-    if (nblk > 0) {
-      const u64 c0 = lane < nblk ? crow[lane] : 0;
-      c_next = 32 + lane < nblk ? crow[32 + lane] : 0;
-      key = chain_chunk<32>(parent, c0, lane, nblk < 32 ? nblk : 32);
-    }
-    for (int base = 0; base < nblk; base += 32) {
-      const int j = base + lane;
-      const bool active = j < nblk;
-      ProbeWindow w;
-      if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
-      u64 next_key = 0;
-      if (base + 32 < nblk) {                                       // ... while the next chunk is chained
-        const u64 cn = c_next;
-        c_next = base + 64 + lane < nblk ? crow[base + 64 + lane] : 0;
-        u64 p = __shfl_sync(FULL, key, 31);
-        const int left = nblk - base - 32;
-        next_key = chain_chunk<32>(p, cn, lane, left < 32 ? left : 32);
-      }
-      if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
-      n_hashed = nblk < base + 32 ? nblk : base + 32;
-      u32 id = NO_ID;
-      if (active) {
-        u32 visited;
-        id = probe_finish(st.table, st.slots, key, w, &visited);
-        probes += 1;
-        visited_sum += visited;
-      }
-      const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
-      const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);
-      const bool hit = active && lane < nf;
-      const unsigned hm = __ballot_sync(FULL, hit);
-      if (hit) {
-        ids_out[r * max_blocks + j] = (int)id;
-        const bool touch = !(flags & F_NO_TOUCH);
-        if (touch && st.policy == 0) st.m_last[id] = epoch;
-        if ((flags & F_PIN) || (touch && st.policy)) {
-          const unsigned same = __match_any_sync(hm, id);            // ids of one request are distinct: groups of one
-          if (lane == __ffs(same) - 1) {
-            const u32 cnt = (u32)__popc(same);
-            if (flags & F_PIN) atomicAdd(&st.m_ref[id], cnt);
-            if (touch && st.policy) touch_block(st, id, epoch, inflation, cnt);
-          }
-        }
-      }
-      m += nf;
-      if (nf < 32) break;
-      key = next_key;
-    }
-    if (lane == 0) { matched[r] = m; hashed[r] = (u32)n_hashed; s_m = m; }
-    u32 qb = lane == 0 ? (u32)nblk : 0, mb = lane == 0 ? (u32)m : 0;
-    probes = __reduce_add_sync(FULL, probes);
-    visited_sum = __reduce_add_sync(FULL, visited_sum);
-    qb = __reduce_add_sync(FULL, qb);
-    mb = __reduce_add_sync(FULL, mb);
-    if (lane < 4) {
-      const u32 v = lane == 0 ? qb : lane == 1 ? probes : lane == 2 ? visited_sum : mb;
-      if (v) atomicAdd(&st.ctrl->lookup_stripes[r % LOOKUP_STRIPES][lane], (u64)v);
-    }
+    const int m = chain_probe_request(st, crow, nblk, r, max_blocks, flags, epoch, matched, ids_out, hashed, nullptr, 0, lane);
+    if (lane == 0) s_m = m;
   }
   __syncthreads();
   const int m = s_m;

@@ -13,6 +13,7 @@
 #include "insert.cuh"
 #include "evict.cuh"
 #include "promote.cuh"
+#include "fused.cuh"
 
 using namespace pts;
 
@@ -23,7 +24,7 @@ inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
   u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, m_flight, ring[2], ctrl, blocked, sort[2], hist, tile_stats, room, desc,
-      keys, eslot, cta_sums, prefix, promo_first, promo_cnt, heads, links, desc_tier, desc_host, total;
+      keys, eslot, cta_sums, prefix, promo_first, promo_cnt, heads, links, desc_tier, desc_host, progress, total;
 };
 
 constexpr u32 MAX_COOP_GRID = 256;      // cooperative kernels use at most this many CTAs (and at most one per SM)
@@ -72,6 +73,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.links = take(M * sizeof(int2));
   L.desc_tier = take((u64)c->hbm_blocks * sizeof(int2));
   L.desc_host = take((c->host_blocks ? (M < c->host_blocks ? M : (u64)c->host_blocks) : 1) * sizeof(int2));
+  L.progress = take((u64)FUSED_MAX_REQUESTS * 8);
   L.total = o;
   return L;
 }
@@ -101,13 +103,16 @@ struct ptstore {
   int2* links;           // fetch: destination list nodes, one per (request, block) entry
   int2* desc_tier;       // demotion: {HBM id, host id} pairs
   int2* desc_host;       // fetch: descriptors of distinct host-tier source blocks
+  u64* progress;         // fused lookup + gather: one progress word per request
+  int fused_smem_set;    // dynamic shared memory already granted to the fused kernel
   int host_ctas;         // grid of the copies that run at host-link speed
   cudaStream_t tier_stream;   // side stream of the asynchronous demotion copy (created on first use)
   cudaEvent_t ev_meta, ev_copy;
   bool tier_ready, tier_pending;
   u32 flight_seq;        // tag of the demotion copy that may still be running (valid while tier_pending)
   u32 fetch_seq;         // sequence number of the last fetch call (tags the list heads; never 0)
-  u32 coop_seq;          // cooperative launches so far (selects the barrier counter)
+  u32 coop_seq;          // cooperative launches with grid barriers so far (selects the barrier counter)
+  u32 gather_seq;        // launches of the fused lookup + gather so far (the tag of its progress words)
   u32 wait_limit;        // polls per bounded wait in the copy kernels' main loop
   // the batch whose chained keys the last lookup left in `keys` / `prefix` (for ptstore_insert_after_lookup)
   const void* lk_tokens; const void* lk_offsets; int lk_R, lk_max_blocks; bool lk_valid;
@@ -162,12 +167,14 @@ Paged to_paged(const ptstore_paged_cache_t* pc) {
   return p;
 }
 
-// a kernel whose CTAs wait for one another at grid-wide barriers: all of them must be resident at once
+// A kernel whose CTAs wait for one another: all of them must be resident at once.  Kernels that meet at grid-wide barriers
+// are numbered by coop_seq, which selects the barrier's counter, and every one of them clears the counter of a later launch,
+// so a kernel that has no barrier must not take a number from that sequence: it gets its own (`barrier` false).
 template <typename Kernel, typename Args>
-int launch_coop(ptstore* h, Kernel kernel, int grid, int threads, Args& args, cudaStream_t s) {
-  args.launch_seq = ++h->coop_seq;
+int launch_coop(ptstore* h, Kernel kernel, int grid, int threads, Args& args, cudaStream_t s, size_t smem = 0, bool barrier = true) {
+  args.launch_seq = barrier ? ++h->coop_seq : ++h->gather_seq;
   void* params[2] = {&h->st, &args};
-  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), params, 0, s);
+  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), params, smem, s);
   h->launches += 1;
   if (e != cudaSuccess) { (void)cudaGetLastError(); h->last_cuda = (int)e; return PTSTORE_E_CUDA; }
   return PTSTORE_OK;
@@ -453,6 +460,50 @@ int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32
   }
 }
 
+// A handful of long prompts, HBM tier only, default copy ring: lookup and gather as one cooperative launch in which the
+// copies of a prompt's first blocks start while its hash chain is still running.  Not taken when the caller asked for
+// events around the copy kernel (there is no separate one).
+bool fused_small_batch(const ptstore* h, int R, int max_blocks) {
+  return split_path(h, R, max_blocks) && R <= FUSED_MAX_REQUESTS && h->cfg.host_blocks == 0 && !(h->cfg.flags & PTSTORE_COPY_VECTOR) &&
+         ((h->cfg.flags >> 16) & 0xFu) == 0 && ((h->cfg.flags >> 20) & 0xFFu) == 0 && h->time_before == nullptr;
+}
+
+int launch_lookup_gather(ptstore* h, const int32_t* tokens, const int64_t* offsets, int R, int max_blocks, u32 flags,
+                         const ptstore_paged_cache_t* dst, const int32_t* block_tables, int32_t* matched, int32_t* ids, cudaStream_t s) {
+  const BulkVariant v = auto_bulk(h->st.chunk_bytes);
+  const int smem = v.stages * v.stage_bytes;
+  if (smem > h->fused_smem_set) {
+    if (cudaFuncSetAttribute(lookup_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      h->last_cuda = (int)cudaGetLastError();
+      return PTSTORE_E_CUDA;
+    }
+    h->fused_smem_set = smem;
+  }
+  const u32 ppc = (u32)((h->st.chunk_bytes + v.stage_bytes - 1) / v.stage_bytes);
+  const u32 per_block = 2u * h->st.layers * ppc;
+  FusedArgs a = {};
+  a.tokens = tokens;
+  a.offsets = reinterpret_cast<const long long*>(offsets);
+  a.R = R; a.max_blocks = max_blocks; a.flags = flags; a.epoch = h->epoch;
+  a.matched = matched; a.ids_out = ids;
+  a.scratch = h->keys; a.hashed = h->prefix;
+  a.bt = block_tables;
+  a.pc = to_paged(dst);
+  a.progress = h->progress;
+  if (++h->fetch_seq == 0) {          // keep the fetch calls' alternation of counters (and their tag wrap) in step
+    const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
+    if (cudaMemsetAsync(h->heads, 0, N * 8, s) != cudaSuccess || cudaMemsetAsync(h->st.ctrl->f_pairs, 0, 6 * sizeof(u32), s) != cudaSuccess) {
+      h->last_cuda = (int)cudaGetLastError();
+      return PTSTORE_E_CUDA;
+    }
+    h->fetch_seq = 1;
+  }
+  a.fetch_seq = h->fetch_seq;
+  a.tune = {v.stages, v.stage_bytes, (int)(per_block >= 4 ? per_block / 4 : per_block), 0, h->wait_limit};
+  h->lk_tokens = tokens; h->lk_offsets = offsets; h->lk_R = R; h->lk_max_blocks = max_blocks; h->lk_valid = true;
+  return launch_coop(h, lookup_gather_kernel, h->coop_grid, LONG_THREADS, a, s, (size_t)smem, false);
+}
+
 template <int L>
 int launch_insert(ptstore* h, InsertArgs& a, int grid, cudaStream_t s) { return launch_coop(h, insert_kernel<L>, grid, INS_THREADS, a, s); }
 
@@ -528,6 +579,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->links = reinterpret_cast<int2*>(w + lay.links);
   h->desc_tier = reinterpret_cast<int2*>(w + lay.desc_tier);
   h->desc_host = reinterpret_cast<int2*>(w + lay.desc_host);
+  h->progress = reinterpret_cast<u64*>(w + lay.progress);
   h->host_ctas = 32;     // a few CTAs saturate the host link; a small grid leaves the SMs to kernels that run beside it
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -537,7 +589,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
   store_init_kernel<<<grid_for((long long)cfg->hbm_blocks + cfg->host_blocks, 256, cap), 256, 0, s>>>(st, h->heads);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
-  ctrl_init_kernel<<<1, 1, 0, s>>>(st);
+  ctrl_init_kernel<<<1, 1, 0, s>>>(st, h->progress, FUSED_MAX_REQUESTS);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
   h->launches = 3;
   *out = h;
@@ -598,6 +650,7 @@ int ptstore_lookup_fetch(ptstore_t* h, const int32_t* tokens, const int64_t* off
   h->epoch += 1;
   if (R == 0) return PTSTORE_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (fused_small_batch(h, R, max_blocks)) return launch_lookup_gather(h, tokens, offsets, R, max_blocks, flags, dst, block_tables, matched_blocks, block_ids, s);
   FetchLink fl;
   rc = next_fetch_link(h, dst, block_tables, s, &fl);
   if (rc) return rc;

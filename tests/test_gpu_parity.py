@@ -689,24 +689,108 @@ def test_lookup_fetch_equals_lookup_then_fetch(name, mk):
     p.close()
 
 
-@pytest.mark.parametrize("host,policy", [(0, "lru"), (20, "lru"), (20, "gdsf")])
-def test_fused_step_lockstep(host, policy):
+@pytest.mark.parametrize("policy", ["lru", "gdsf"])
+def test_small_batch_of_long_prompts_is_looked_up_and_gathered_in_one_launch(policy):
+    """Up to 16 prompts of more than 32 blocks: one cooperative launch in which the copy CTAs follow the lookups' progress.
+    Match lengths of zero, inside a chunk of 32, on chunk borders and the whole prompt; prompts that share blocks; chunks
+    that split into several pieces and units; pinning; then the same batches one request too wide (two launches)."""
+    Pair, dev, G = _imports()
+    rng = np.random.default_rng(31)
+    for sh, mbs in ((W.KVShape(2, 1, 8, 2), (33, 100, 260)), (W.KVShape(2, 8, 136, 16), (70,))):   # chunks of 32 B and of 34 KiB
+        B = sh.block_tokens
+        pool = 900
+        p = Pair(sh, pool, max_requests=20, max_batch_blocks=20 * 260, policy=policy)
+        for mb in mbs:
+            base = rng.integers(0, 60000, size=mb * B, dtype=np.int32)
+            other = rng.integers(0, 60000, size=mb * B, dtype=np.int32)
+            stored = min(mb, 70)
+            for doc in (base[: stored * B], other[: (stored // 2) * B]):
+                nb = len(doc) // B
+                tab = np.full((1, mb), -1, dtype=np.int32); tab[0, :nb] = rng.permutation(nb + 2)[:nb]
+                p.insert([doc], mb, W.random_kv_cache(mb, sh, nb + 2), tab)
+            fresh = lambda n: rng.integers(60000, 99999, size=max(n, 0) * B, dtype=np.int32)
+            cuts = [k for k in (0, 1, 31, 32, 33, 64, stored) if k <= stored]
+            batch = [np.concatenate([base[: k * B], fresh(mb - k)])[: mb * B] for k in cuts]
+            batch += [base, other, other[: 5 * B], base[: 40 * B + B // 2], fresh(2)]
+            for R in (1, 3, len(batch), 16, 17):
+                seqs = [batch[i % len(batch)] for i in range(R)]
+                upper = [min(len(s) // B, mb) for s in seqs]
+                nd = sum(upper) + 3
+                bt = _tables_for(rng, upper, R, mb, nd)
+                dst = [np.full((2, nd, sh.chunk_bytes), 0x5A, dtype=np.uint8) for _ in range(sh.layers)]
+                before = p.g.launch_count()
+                mo, io = p.lookup_fetch(seqs, mb, dst, bt, flags=R % 2)
+                assert p.g.launch_count() - before == (1 if R <= 16 else 2)
+                if R >= len(batch):
+                    assert mo[: len(cuts)].tolist() == cuts
+                if R % 2:
+                    p.release(io, mo)
+                assert p.check_status() == 0
+            # an out-of-range destination and a negative one: those entries are skipped, the first is flagged, the rest copied
+            seqs = [base, other]
+            upper = [mb, mb]
+            nd = 2 * mb + 1
+            bt = _tables_for(rng, upper, 2, mb, nd)
+            bt[0, 3] = nd + 9
+            bt[1, 0] = -1
+            dst = [np.full((2, nd, sh.chunk_bytes), 0x5A, dtype=np.uint8) for _ in range(sh.layers)]
+            p.lookup_fetch(seqs, mb, dst, bt)
+            assert p.check_status() == G.S_BOUNDS
+        s = p.check_counts()
+        assert s.blocks_fetched[0] == s.blocks_matched
+        p.close()
+
+
+def test_one_launch_lookup_gather_gives_up_on_a_wait_that_runs_out():
+    """One poll per copy wait: the fused kernel's copiers give up at their first wait, drain and return; S_TIMEOUT is
+    raised, matched lengths and ids are still right, and with the limit restored the same call is byte-exact."""
+    Pair, dev, G = _imports()
+    sh = W.LLAMA3_8B
+    B = sh.block_tokens
+    rng = np.random.default_rng(4)
+    mb = 40
+    p = Pair(sh, 48, max_requests=4, max_batch_blocks=4 * mb)
+    doc = rng.integers(0, 1000, size=36 * B, dtype=np.int32)
+    tab = np.full((1, mb), -1, dtype=np.int32); tab[0, :36] = np.arange(36)
+    p.insert([doc], mb, W.random_kv_cache(3, sh, 36), tab)
+    toks, offs = W.ragged([doc, doc[: 20 * B]])
+    bt = np.full((2, mb), -1, dtype=np.int32); bt[0, :36] = np.arange(36); bt[1, :20] = np.arange(36, 56)
+    mo, io = p.o.lookup(toks, offs, mb, 0)
+    cache = G.PagedKV(sh.layers, 56, sh.chunk_bytes)
+    p.g.set_wait_limit(1)
+    before = p.g.launch_count()
+    mg, ig = p.g.lookup_fetch(dev(toks), dev(offs), mb, cache, dev(bt), 0)
+    assert p.g.launch_count() - before == 1
+    assert p.g.status() & G.S_TIMEOUT
+    assert (mg.cpu().numpy() == mo).all() and (ig.cpu().numpy() == io).all()
+    p.g.set_wait_limit(0)
+    dst = [np.zeros((2, 56, sh.chunk_bytes), dtype=np.uint8) for _ in range(sh.layers)]
+    p.lookup_fetch([doc, doc[: 20 * B]], mb, dst, bt)
+    assert p.check_status() == 0
+    p.check_counts()
+    p.close()
+
+
+@pytest.mark.parametrize("host,policy,mb", [(0, "lru", 12), (20, "lru", 12), (20, "gdsf", 12), (0, "lru", 40), (0, "gdsf", 40)])
+def test_fused_step_lockstep(host, policy, mb):
     """A serving loop made of the fused calls only: lookup_fetch(PIN) -> reserve -> insert -> release, random batches,
-    compared call by call; with a host tier the reserve demotes (synchronously or with the copy on the side stream)."""
+    compared call by call; with a host tier the reserve demotes (synchronously or with the copy on the side stream).
+    With 40 blocks per prompt and no host tier the lookup_fetch is the single cooperative launch, between the cooperative
+    kernels of reserve and insert, for enough steps that their barrier counters are reused many times."""
     Pair, dev, G = _imports()
     sh = W.KVShape(2, 1, 8, 2)
     B = 2
     for seed in range(4):
         rng = np.random.default_rng(700 + seed)
-        p = Pair(sh, 36, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * 12, table_slots=307, policy=policy)
+        p = Pair(sh, 36 if mb == 12 else 150, host_blocks=host, salt=seed, max_requests=8, max_batch_blocks=8 * mb, table_slots=307 if mb == 12 else 1201,
+                 policy=policy)
         seqs = []
-        for step in range(50):
+        for step in range(50 if mb == 12 else 80):
             base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.75 else np.zeros(0, dtype=np.int32)
             cut = int(rng.integers(0, len(base) + 1))
-            s = np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(1, 10)), dtype=np.int32)])[:24]
+            s = np.concatenate([base[:cut], rng.integers(0, 3, size=int(rng.integers(1, 10 if mb == 12 else 50)), dtype=np.int32)])[: 2 * mb]
             seqs.append(s)
             batch = [seqs[int(rng.integers(0, len(seqs)))] for _ in range(int(rng.integers(1, 6)))] + [s]
-            mb = 12
             upper = [len(x) // B for x in batch]
             nd = sum(upper) + 2
             bt = _tables_for(rng, upper, len(batch), mb, nd)
@@ -724,6 +808,62 @@ def test_fused_step_lockstep(host, policy):
         p.check_pools()
         p.check_counts()
         p.close()
+
+
+def test_few_long_full_hit_prompts_with_little_slack_lockstep():
+    """The latency workload in small: 32 stored documents of 256 blocks, prompts of a whole document plus 4 fresh blocks,
+    batches of 1, 4 and 16, a pool with so little slack that room is made all the time (at one point the free blocks are
+    exactly what the batch needs).  Every step is lookup_fetch(PIN) -> reserve -> insert_after_lookup -> release, compared
+    call by call; the insert and evict kernels run with several CTAs here, between the one-launch lookup + gather."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 2)
+    B, n_docs, doc_blocks, suf_blocks = 2, 32, 256, 4
+    mb = doc_blocks + suf_blocks
+    pool = n_docs * doc_blocks + 8 * n_docs * suf_blocks
+    rng = np.random.default_rng(77)
+    p = Pair(sh, pool, max_requests=16, max_batch_blocks=16 * mb)
+    docs = [rng.integers(0, 128256, size=doc_blocks * B, dtype=np.int32) for _ in range(n_docs)]
+    for k in range(0, n_docs, 16):
+        part = docs[k:k + 16]
+        bt = np.arange(len(part) * mb, dtype=np.int32).reshape(len(part), mb)
+        p.insert(part, mb, W.random_kv_cache(k, sh, len(part) * mb), bt)
+    next_doc = 0
+    for b, n_steps in ((1, 70), (4, 40), (16, 30)):
+        for step in range(n_steps):
+            batch = []
+            for _ in range(b):
+                batch.append(np.concatenate([docs[next_doc % n_docs], rng.integers(0, 128256, size=suf_blocks * B, dtype=np.int32)]))
+                next_doc += 1
+            bt = rng.permutation(b * mb).astype(np.int32).reshape(b, mb)
+            dst = W.random_kv_cache(1000 * b + step, sh, b * mb)
+            mo, io = p.lookup_fetch(batch, mb, dst, bt, flags=1)
+            assert (mo == doc_blocks).all()
+            p.reserve(b * mb, mo, headroom=64 if b < 16 else 0)
+            _, newb = p.insert(batch, mb, dst, bt, after_lookup=bool(step % 2))      # resumed behind the lookup's keys, or hashed anew
+            assert (newb == suf_blocks).all()
+            p.release(io, mo)
+            assert p.check_status() == 0
+        p.check_pools()
+        p.check_counts()
+    assert p.g.resumed_inserts() == 70
+    # uneven work for the insert's CTAs (long and one-block prompts by turns, hashed anew): one CTA is through its hash
+    # chains long before the other, so the phases only come out right if the grid-wide barriers between them hold
+    for step in range(24):
+        batch = []
+        for i in range(5):
+            fresh = rng.integers(0, 128256, size=(suf_blocks if i % 2 == 0 else 1) * B, dtype=np.int32)
+            batch.append(np.concatenate([docs[next_doc % n_docs], fresh]) if i % 2 == 0 else fresh)
+            next_doc += 1
+        bt = rng.permutation(5 * mb).astype(np.int32).reshape(5, mb)
+        dst = W.random_kv_cache(5000 + step, sh, 5 * mb)
+        mo, io = p.lookup_fetch(batch, mb, dst, bt, flags=1)
+        p.reserve(5 * mb, mo, headroom=8)
+        p.insert(batch, mb, dst, bt)
+        p.release(io, mo)
+        assert p.check_status() == 0
+    p.check_pools()
+    p.check_counts()
+    p.close()
 
 
 def test_insert_after_lookup_resumes_behind_the_lookups_keys():
