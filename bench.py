@@ -709,15 +709,21 @@ def run_latency(args):
     build()
     sampler = ClockSampler(0)
     sampler.start()
-    rec = latency_record(args, torch, iters=max(args.steps, 10))
+    kw = {}
+    if args.batch:                        # a small case (for a profiler): one batch size, fewer stored documents
+        kw["batches"] = (args.batch,)
+    if args.docs:
+        kw["n_docs"] = args.docs
+    rec = latency_record(args, torch, iters=max(args.steps, 10), **kw)
     clocks = sampler.stop()
-    b1 = rec["batch1"]
+    b1 = rec["batch%d" % (args.batch or 1)]
     peak, kind = measured_peak()
     out = {"metric": "prefix-hit KV fetch GB/s", "value": b1["gbps"], "unit": "GB/s", "n_gpus": 1, "steps": rec["config"]["iters"], "warmup": 8,
            "ms_per_step": round(b1["step_us"] / 1e3, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
-           "data": "synthetic", "config": dict(rec["config"], workload="latency_llama3_8b_4k_prompt_full_hit_batch1_4_16", l2="512 MiB of KV per prompt: larger than L2"),
+           "data": "synthetic", "config": dict(rec["config"], workload="latency_llama3_8b_4k_prompt_full_hit_batch" + "_".join(str(b) for b in kw.get("batches", (1, 4, 16))),
+                          l2="512 MiB of KV per prompt: larger than L2"),
            "latency": rec, "gpu_launches": int(b1["launches_per_step"] * rec["config"]["iters"]), "clocks": clocks,
-           "roofline": {"bound": "hbm", "kernel": "whole batch-1 step", "achieved": b1["gbps"], "peak": peak, "unit": "GB/s",
+           "roofline": {"bound": "hbm", "kernel": "whole batch-%d step" % (args.batch or 1), "achieved": b1["gbps"], "peak": peak, "unit": "GB/s",
                         "frac": round(b1["gbps"] / peak, 4), "traffic": None, "peak_kind": kind + " (plain copy, read+write)"}}
     print(json.dumps(out), flush=True)
 

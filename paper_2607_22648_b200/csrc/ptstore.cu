@@ -499,7 +499,9 @@ int launch_lookup_gather(ptstore* h, const int32_t* tokens, const int64_t* offse
     h->fetch_seq = 1;
   }
   a.fetch_seq = h->fetch_seq;
-  a.tune = {v.stages, v.stage_bytes, (int)(per_block >= 4 ? per_block / 4 : per_block), 0, h->wait_limit};
+  // units of an eighth of a block: with so few blocks the last units decide the time (measured on B200, batch 1 / 4 / 16,
+  // whole step: a quarter 210 / 712 / 2681 us, an eighth 207 / 705 / 2681, a sixteenth 209 / 724 / 2764)
+  a.tune = {v.stages, v.stage_bytes, (int)(per_block >= 8 ? per_block / 8 : per_block), 0, h->wait_limit};
   h->lk_tokens = tokens; h->lk_offsets = offsets; h->lk_R = R; h->lk_max_blocks = max_blocks; h->lk_valid = true;
   return launch_coop(h, lookup_gather_kernel, h->coop_grid, LONG_THREADS, a, s, (size_t)smem, false);
 }
