@@ -173,11 +173,13 @@ def test_large_blocks_of_1024_tokens():
     srv.close()
 
 
-@pytest.mark.parametrize("host,policy,shape", [(0, "lru", "long16"), (4000, "gdsf", "long4"), (0, "gdsf", "short1500"), (20000, "lru", "short1100")])
+@pytest.mark.parametrize("host,policy,shape", [(0, "lru", "long16"), (4000, "gdsf", "long4"), (0, "gdsf", "long8"), (0, "gdsf", "short1500"),
+                                               (20000, "lru", "short1100")])
 def test_medium_serving_loops_where_cooperative_kernels_span_several_ctas(host, policy, shape):
     """Medium sizes between the small lock-step tests and the full-size ones: eviction over 3,000-15,000 block ids (6-30 CTAs
     meeting at grid barriers), insert metadata over 2,500-20,000 elements (3-20 CTAs), long prompts (one CTA per request)
-    and thousands of short ones (sub-warps, lists linked inside the chunk loop); two thirds of the steps use the fused calls,
+    and thousands of short ones (sub-warps, lists linked inside the chunk loop; "long8": 12 prompts and no host tier, so the
+    fused call is the single lookup + gather launch); two thirds of the steps use the fused calls,
     the rest the separate ones with promotion and asynchronous demotion; table rebuilds happen every few steps."""
     from tests.serving import LockstepServing
     if shape.startswith("long"):
