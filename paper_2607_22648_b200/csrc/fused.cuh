@@ -9,10 +9,12 @@
 // block as soon as its request's progress word says it is matched.  The CTAs of a cooperative launch are all resident,
 // so the copiers may wait for the lookups; every wait is bounded (S_TIMEOUT, then drain and return).
 //
-// Work units are dealt from an atomic counter in a fixed order: unit u = ((j * R + r) * U + q) is part q of block j of
-// request r, so early blocks, which are matched first, are handed out first and a copier rarely has to wait.  Every
-// (request, block) entry is copied on its own - no sharing of reads between requests that name the same pool block -
-// which is why the host only takes this path for small batches.
+// Work units - part q of block j of request r - are dealt per request: every request has a counter of units taken (in the
+// order of its blocks, so the blocks that match first are copied first), and a copier goes round the requests, one unit
+// at a time, dropping a request once its counter has passed the end of what matched.  A batch of one long prompt and
+// fifteen that miss therefore costs a copier fifteen wasted counter reads, not fifteen of every sixteen.  Every (request,
+// block) entry is copied on its own - no sharing of reads between requests that name the same pool block - which is why
+// the host only takes this path for small batches.
 #pragma once
 #include "common.cuh"
 #include "lookup.cuh"
@@ -35,9 +37,11 @@ struct FusedArgs {
   u32* hashed;
   const int* bt;            // destination block tables
   Paged pc;
-  u64* progress;            // [R] progress words
-  u32 fetch_seq;            // sequence number of this call among the handle's fetch calls: selects the work counter
-                            // (zero at launch) and, as in every fetch, the next call's scalars are cleared here
+  u64* progress;            // [FUSED_MAX_REQUESTS] progress words
+  u32* taken;               // [FUSED_MAX_REQUESTS] units of each request handed out so far; request r's is reset by the CTA
+                            // that looks r up, before that CTA's first progress word of this launch
+  u32 fetch_seq;            // sequence number of this call among the handle's fetch calls: as in every fetch, the next
+                            // call's list scalars are cleared here
   BulkTune tune;
   u32 launch_seq;           // this kernel's own launch count, from 1: the tag of the progress words
 };
@@ -57,12 +61,12 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
     seq_only.seq = a.fetch_seq;
     link_prepare_next(st, seq_only);
   }
-  u32* const work_counter = &st.ctrl->f_work[a.fetch_seq & 1u];
   // ---- the lookup of request blockIdx.x ---------------------------------------------------------------------------------
   if ((int)blockIdx.x < R) {
     const long long r = blockIdx.x;
     const int nblk = full_blocks(a.offsets, (int)r, st.block_tokens, max_blocks);
     u64* crow = a.scratch + r * max_blocks;
+    if (threadIdx.x == 0) a.taken[r] = 0;        // ordered before this thread's release of the first progress word
     {
       const int* t0 = a.tokens + a.offsets[r];
       for (int j = threadIdx.x; j < nblk; j += LONG_THREADS) crow[j] = content_block(t0 + (long long)j * st.block_tokens, st.block_tokens);
@@ -94,53 +98,49 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   fence_async_smem();
 
-  // what is known of each request: matched so far, and whether that is final
-  int known[FUSED_MAX_REQUESTS];
-  bool final_[FUSED_MAX_REQUESTS];
-#pragma unroll
-  for (int r = 0; r < FUSED_MAX_REQUESTS; ++r) { known[r] = 0; final_[r] = false; }
+  // what this copier knows of each request: blocks matched so far, and whether that is final (used by thread 0 only)
+  __shared__ int s_known[FUSED_MAX_REQUESTS];
+  __shared__ int s_final[FUSED_MAX_REQUESTS];
+  for (int r = 0; r < FUSED_MAX_REQUESTS; ++r) { s_known[r] = 0; s_final[r] = 0; }
   bool ok = true;
-  // waits until entry (r, j) is known to exist (true) or not to (false)
-  auto entry_exists = [&](int r, int j) -> bool {
-    int kn = 0; bool fin = false;
-#pragma unroll
-    for (int i = 0; i < FUSED_MAX_REQUESTS; ++i) if (i == r) { kn = known[i]; fin = final_[i]; }
+  // Reads request r's progress word until it covers block j or is final (j < 0: until it carries this launch's tag with
+  // something to copy, or is final).  False when the wait ran out.
+  auto await = [&](int r, int j) -> bool {
     u32 polls = 0;
-    while (j >= kn && !fin) {
+    while (true) {
       u64 v;
       asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(a.progress + r) : "memory");
-      if ((u32)(v >> 32) == tag) { kn = (int)(v & 0x7FFFFFFFull); fin = (v & 0x80000000ull) != 0; }
-      if (j < kn || fin) break;
-      if (++polls >= PROGRESS_POLL_LIMIT) { ok = false; raise(st, S_TIMEOUT); fin = true; break; }
+      if ((u32)(v >> 32) == tag) {
+        const int kn = (int)(v & 0x7FFFFFFFull);
+        const int fin = (v & 0x80000000ull) != 0;
+        s_known[r] = kn; s_final[r] = fin;
+        if (fin || (j < 0 ? kn > 0 : j < kn)) return true;
+      }
+      if (++polls >= PROGRESS_POLL_LIMIT) { ok = false; raise(st, S_TIMEOUT); return false; }
       __nanosleep(64);
     }
-#pragma unroll
-    for (int i = 0; i < FUSED_MAX_REQUESTS; ++i) if (i == r) { known[i] = kn; final_[i] = fin; }
-    return j < kn;
-  };
-  auto all_final_below = [&](int j) -> bool {      // every request is final and none reaches block j
-    bool done = true;
-#pragma unroll
-    for (int i = 0; i < FUSED_MAX_REQUESTS; ++i) if (i < R) done = done && final_[i] && known[i] <= j;
-    return done;
   };
 
-  // generator of pieces: takes units from the counter
+  // generator of pieces: goes round the requests that may still have units and takes one unit at a time
+  u32 alive = R >= 32 ? 0xFFFFFFFFu : ((1u << R) - 1u);
+  int cur = (int)(blockIdx.x % (unsigned)R);
   u32 in_unit = 0, unit_pieces = 0, ls = 0, piece = 0;
   const unsigned char* src_block = nullptr;
   u32 dst_block = 0;
   bool exhausted = false;
   auto next_unit = [&]() -> bool {                  // positions the cursor on the next unit that exists
-    while (ok) {
-      const u64 u = (u64)atomicAdd(work_counter, 1u);
-      const u32 q = (u32)(u % U);
-      const u64 t = u / U;
-      const int r = (int)(t % (u64)R), j = (int)(t / (u64)R);
-      if (j >= max_blocks) return false;
-      if (!entry_exists(r, j)) {
-        if (all_final_below(j)) return false;
-        continue;
-      }
+    while (ok && alive) {
+      int r = cur;
+      while (!((alive >> r) & 1u)) r = r + 1 == R ? 0 : r + 1;
+      cur = r + 1 == R ? 0 : r + 1;
+      // the counter of r may be touched only after a progress word of this launch has been seen (it is reset before)
+      if (s_known[r] == 0 && !s_final[r] && !await(r, -1)) return false;
+      if (s_known[r] == 0) { alive &= ~(1u << r); continue; }            // final with nothing matched
+      const u32 u = atomicAdd(a.taken + r, 1u);
+      const int j = (int)(u / U);
+      const u32 q = u - (u32)j * U;
+      if (j >= s_known[r] && !s_final[r] && !await(r, j)) return false;
+      if (j >= s_known[r]) { alive &= ~(1u << r); continue; }            // final and shorter: nothing left of r
       const long long e = (long long)r * max_blocks + j;
       const int id = __ldcg(a.ids_out + e), cb = a.bt[e];      // ids are written during this launch: not through L1
       if (id < 0 || (u32)id >= st.n[0] || cb < 0 || (u32)cb >= a.pc.num_blocks) {

@@ -73,7 +73,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.links = take(M * sizeof(int2));
   L.desc_tier = take((u64)c->hbm_blocks * sizeof(int2));
   L.desc_host = take((c->host_blocks ? (M < c->host_blocks ? M : (u64)c->host_blocks) : 1) * sizeof(int2));
-  L.progress = take((u64)FUSED_MAX_REQUESTS * 8);
+  L.progress = take((u64)FUSED_MAX_REQUESTS * 16);      // a progress word and a unit counter per request
   L.total = o;
   return L;
 }
@@ -490,6 +490,7 @@ int launch_lookup_gather(ptstore* h, const int32_t* tokens, const int64_t* offse
   a.bt = block_tables;
   a.pc = to_paged(dst);
   a.progress = h->progress;
+  a.taken = reinterpret_cast<u32*>(h->progress + FUSED_MAX_REQUESTS);
   if (++h->fetch_seq == 0) {          // keep the fetch calls' alternation of counters (and their tag wrap) in step
     const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
     if (cudaMemsetAsync(h->heads, 0, N * 8, s) != cudaSuccess || cudaMemsetAsync(h->st.ctrl->f_pairs, 0, 6 * sizeof(u32), s) != cudaSuccess) {
