@@ -207,8 +207,8 @@ int ptstore_lookup(ptstore_t* st, const int32_t* tokens, const int64_t* offsets,
  * block_tables[r*max_blocks+j] as by ptstore_fetch.  The lookup kernel builds the copy lists itself while it probes,
  * so the pair costs two kernel launches (three with a host tier).  A batch of at most 16 requests of more than 32 blocks
  * against a store without a host tier (default copy engine, no ptstore_time_next_copy pending) is one cooperative launch:
- * the copies of a request's first blocks run while the rest of its hash chain is still being looked up; every (request,
- * block) entry is then copied on its own, also when two requests name the same pool block.
+ * the copies of a request's first blocks run while the rest of its hash chain is still being looked up.  Either way a
+ * pool block named by several entries of the call is read once and written to every destination.
  */
 int ptstore_lookup_fetch(ptstore_t* st, const int32_t* tokens, const int64_t* offsets, int32_t R, int32_t max_blocks,
                          uint32_t flags, const ptstore_paged_cache_t* dst /*host struct*/,

@@ -73,7 +73,7 @@ Layout make_layout(const ptstore_config_t* c) {
   L.links = take(M * sizeof(int2));
   L.desc_tier = take((u64)c->hbm_blocks * sizeof(int2));
   L.desc_host = take((c->host_blocks ? (M < c->host_blocks ? M : (u64)c->host_blocks) : 1) * sizeof(int2));
-  L.progress = take((u64)FUSED_MAX_REQUESTS * 16);      // a progress word and a unit counter per request
+  L.progress = take((u64)FUSED_MAX_REQUESTS * 24);      // per request: two progress words and a unit counter
   L.total = o;
   return L;
 }
@@ -103,7 +103,7 @@ struct ptstore {
   int2* links;           // fetch: destination list nodes, one per (request, block) entry
   int2* desc_tier;       // demotion: {HBM id, host id} pairs
   int2* desc_host;       // fetch: descriptors of distinct host-tier source blocks
-  u64* progress;         // fused lookup + gather: one progress word per request
+  u64* progress;         // fused lookup + gather, per request: lookup progress word, owned-list progress word, unit counter
   int fused_smem_set;    // dynamic shared memory already granted to the fused kernel
   int host_ctas;         // grid of the copies that run at host-link speed
   cudaStream_t tier_stream;   // side stream of the asynchronous demotion copy (created on first use)
@@ -464,7 +464,7 @@ int lookup_impl(ptstore* h, const int32_t* tokens, const int64_t* offsets, int32
 // copies of a prompt's first blocks start while its hash chain is still running.  Not taken when the caller asked for
 // events around the copy kernel (there is no separate one).
 bool fused_small_batch(const ptstore* h, int R, int max_blocks) {
-  return split_path(h, R, max_blocks) && R <= FUSED_MAX_REQUESTS && h->cfg.host_blocks == 0 && !(h->cfg.flags & PTSTORE_COPY_VECTOR) &&
+  return split_path(h, R, max_blocks) && R <= FUSED_MAX_REQUESTS && max_blocks <= FUSED_MAX_BLOCKS && h->cfg.host_blocks == 0 && !(h->cfg.flags & PTSTORE_COPY_VECTOR) &&
          ((h->cfg.flags >> 16) & 0xFu) == 0 && ((h->cfg.flags >> 20) & 0xFFu) == 0 && h->time_before == nullptr;
 }
 
@@ -490,7 +490,10 @@ int launch_lookup_gather(ptstore* h, const int32_t* tokens, const int64_t* offse
   a.bt = block_tables;
   a.pc = to_paged(dst);
   a.progress = h->progress;
-  a.taken = reinterpret_cast<u32*>(h->progress + FUSED_MAX_REQUESTS);
+  a.owned_progress = h->progress + FUSED_MAX_REQUESTS;
+  a.taken = reinterpret_cast<u32*>(h->progress + 2 * FUSED_MAX_REQUESTS);
+  a.owned = h->eslot;                  // scratch of the insert kernel, free between inserts
+  a.owned_src = h->links;              // list nodes of the list-based fetch, which this call replaces
   if (++h->fetch_seq == 0) {          // keep the fetch calls' alternation of counters (and their tag wrap) in step
     const u64 N = (u64)h->cfg.hbm_blocks + h->cfg.host_blocks;
     if (cudaMemsetAsync(h->heads, 0, N * 8, s) != cudaSuccess || cudaMemsetAsync(h->st.ctrl->f_pairs, 0, 6 * sizeof(u32), s) != cudaSuccess) {
@@ -592,7 +595,7 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
   store_init_kernel<<<grid_for((long long)cfg->hbm_blocks + cfg->host_blocks, 256, cap), 256, 0, s>>>(st, h->heads);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
-  ctrl_init_kernel<<<1, 1, 0, s>>>(st, h->progress, FUSED_MAX_REQUESTS);
+  ctrl_init_kernel<<<1, 1, 0, s>>>(st, h->progress, 2 * FUSED_MAX_REQUESTS);
   if (cudaGetLastError() != cudaSuccess) return fail(PTSTORE_E_CUDA);
   h->launches = 3;
   *out = h;

@@ -736,6 +736,22 @@ def test_small_batch_of_long_prompts_is_looked_up_and_gathered_in_one_launch(pol
             dst = [np.full((2, nd, sh.chunk_bytes), 0x5A, dtype=np.uint8) for _ in range(sh.layers)]
             p.lookup_fetch(seqs, mb, dst, bt)
             assert p.check_status() == G.S_BOUNDS
+            # the same where prompts share blocks (read once, written to every prompt that names them): a bad entry of the
+            # lowest prompt and one of a prompt that shares with it are skipped, every other destination is written
+            seqs = [base, base, base[: 10 * B], other, base]
+            upper = [min(len(x) // B, mb) for x in seqs]
+            nd = sum(upper) + 1
+            bt = _tables_for(rng, upper, len(seqs), mb, nd)
+            bt[0, 3] = nd + 9
+            bt[1, 5] = -4
+            bt[4, 5] = nd
+            dst = [np.full((2, nd, sh.chunk_bytes), 0x5A, dtype=np.uint8) for _ in range(sh.layers)]
+            before = p.g.stats()
+            p.lookup_fetch(seqs, mb, dst, bt)
+            assert p.check_status() == G.S_BOUNDS
+            after = p.g.stats()
+            stored_other = min(mb, 70) // 2
+            assert after.blocks_fetched_distinct - before.blocks_fetched_distinct == min(mb, 70) + stored_other   # base's and other's blocks, once each
         s = p.check_counts()
         assert s.blocks_fetched[0] == s.blocks_matched
         p.close()
