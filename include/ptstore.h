@@ -58,7 +58,7 @@ typedef void* ptstore_stream_t;        /* a cudaStream_t; NULL = the legacy defa
 
 /* bits of the device status word (ptstore_status) */
 #define PTSTORE_S_NOSPACE     0x1u   /* insert: HBM free ring ran dry, some blocks were denied */
-#define PTSTORE_S_TABLE_FULL  0x2u   /* insert/rebuild: no free slot found within table_slots probes */
+#define PTSTORE_S_TABLE_FULL  0x2u   /* insert: no free slot found within table_slots probes */
 #define PTSTORE_S_BOUNDS      0x4u   /* a block id or block-table entry was out of range; access skipped */
 #define PTSTORE_S_STATE       0x8u   /* release would have driven a refcount below zero; skipped */
 #define PTSTORE_S_TIMEOUT     0x10u  /* a bounded wait inside a kernel expired (a copy CTA stopped copying, or a grid-wide
@@ -138,7 +138,8 @@ typedef struct {                 /* all counters are cumulative since create */
   uint64_t epoch;                /* lookup + insert calls so far (the LRU clock) */
   uint64_t live_nodes[2];        /* trie nodes per tier right now */
   uint64_t free_blocks[2];       /* free-ring fill per tier right now */
-  uint64_t tombstones;           /* deleted slots not yet reclaimed by a rebuild */
+  uint64_t max_displacement;     /* largest distance from its home slot at which the table has ever placed a key
+                                    (counted from 24 slots up, else 0) */
   uint64_t query_blocks;         /* full blocks presented to lookup */
   uint64_t probes_issued;        /* keys actually searched by lookup */
   uint64_t slots_visited;        /* table slots read by those searches */
@@ -148,7 +149,8 @@ typedef struct {                 /* all counters are cumulative since create */
   uint64_t blocks_denied;
   uint64_t blocks_dropped[2];    /* deleted per tier */
   uint64_t blocks_demoted;       /* HBM -> host */
-  uint64_t rebuilds;
+  uint64_t far_keys;             /* keys placed 24 or more slots from their home slot so far (a lookup of such a key
+                                    takes a second round of loads) */
   uint64_t blocks_promoted;      /* host -> HBM */
   uint64_t gdsf_clock;           /* GDSF policy: largest priority evicted so far */
   uint64_t blocks_fetched_distinct; /* distinct source blocks read by fetch calls: a block named by several requests
@@ -156,7 +158,7 @@ typedef struct {                 /* all counters are cumulative since create */
 } ptstore_stats_t;
 
 /*
- * Bytes of workspace ptstore_create needs for this configuration (table x2, per-block metadata,
+ * Bytes of workspace ptstore_create needs for this configuration (table, per-block metadata,
  * free rings, per-batch scratch).  Only the size fields of cfg are read.  Returns 0 if cfg is invalid.
  * No paper counterpart: the paper couples its store to a pre-registered allocator (Section 5,
  * second paragraph); here the caller pre-allocates instead.

@@ -50,10 +50,10 @@ class PagedCache(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("epoch", C.c_uint64), ("live_nodes", C.c_uint64 * 2), ("free_blocks", C.c_uint64 * 2),
-                ("tombstones", C.c_uint64), ("query_blocks", C.c_uint64), ("probes_issued", C.c_uint64),
+                ("max_displacement", C.c_uint64), ("query_blocks", C.c_uint64), ("probes_issued", C.c_uint64),
                 ("slots_visited", C.c_uint64), ("blocks_matched", C.c_uint64), ("blocks_fetched", C.c_uint64 * 2),
                 ("blocks_inserted", C.c_uint64), ("blocks_denied", C.c_uint64), ("blocks_dropped", C.c_uint64 * 2),
-                ("blocks_demoted", C.c_uint64), ("rebuilds", C.c_uint64), ("blocks_promoted", C.c_uint64), ("gdsf_clock", C.c_uint64), ("blocks_fetched_distinct", C.c_uint64)]
+                ("blocks_demoted", C.c_uint64), ("far_keys", C.c_uint64), ("blocks_promoted", C.c_uint64), ("gdsf_clock", C.c_uint64), ("blocks_fetched_distinct", C.c_uint64)]
 
 
 EXPORTS = ["ptstore_workspace_bytes", "ptstore_create", "ptstore_destroy", "ptstore_hash", "ptstore_lookup",

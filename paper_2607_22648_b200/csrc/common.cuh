@@ -12,15 +12,33 @@ typedef unsigned int u32;
 constexpr unsigned FULL = 0xFFFFFFFFu;   // all lanes of a warp
 
 // ---- hash table slot ------------------------------------------------------------------------------
-// 16 bytes, loaded with one 128-bit access.  key 0 = never used, key 1 = deleted.
-// id = NO_ID while a slot has been claimed by an insert that has not assigned its block yet.
+// 16 bytes, loaded with one 128-bit access.  key 0 = empty (keys 0 and 1 are never produced by the hash).
+// Keys are placed by linear probing (the first empty slot at or after the home slot), but a lookup does not walk the run:
+// `hop` of a slot says where the keys that have THIS slot as their home sit -
+//   bit d, d = 0..23          : slot home + d
+//   bit 24 + g, g = 0..6      : somewhere in the 32 slots from home + 24 + 32 g
+//   bit 31                    : 248 or more slots away (every slot from there to the largest distance ever used is compared)
+// - so a lookup reads the home slot with its neighbours and then exactly the flagged slots, and a miss costs the same one
+// round trip as a hit (at load factor 0.7 about one key in 250 sits 24 or more slots from home).  Nothing depends on runs
+// being unbroken, so a deleted key simply leaves an empty slot: no deleted markers, no rebuilds.  Deleting clears an exact
+// bit; a group bit or the far bit is cleared by the next lookup that follows it and finds no key of this home there.
+// id: the block of the node; NO_ID in an empty slot; ID_PENDING | r while an insert that has claimed the slot in this
+// call has not been granted its block yet (r = lowest request index that presented the key).
 struct __align__(16) Slot {
   u64 key;
   u32 id;
-  u32 aux;      // insert only: lowest request index that presented this new key
+  u32 hop;
 };
 constexpr u64 KEY_EMPTY = 0ull;
-constexpr u64 KEY_TOMB = 1ull;
+constexpr u32 ID_PENDING = 0x80000000u;     // block ids are below this
+constexpr u32 HOP_EXACT = 24;               // displacements below this have a bit of their own
+constexpr u32 HOP_GROUP = 32;               // slots per group bit
+constexpr u32 HOP_GROUPS = 7;
+constexpr u32 HOP_FAR_FROM = HOP_EXACT + HOP_GROUP * HOP_GROUPS;   // 248
+constexpr u32 HOP_FAR = 0x80000000u;        // bit 31 of hop
+__host__ __device__ __forceinline__ u32 hop_bit(u32 d) {
+  return d < HOP_EXACT ? 1u << d : d < HOP_FAR_FROM ? 1u << (HOP_EXACT + (d - HOP_EXACT) / HOP_GROUP) : HOP_FAR;
+}
 constexpr u32 NO_ID = 0xFFFFFFFFu;
 constexpr u32 NO_SLOT = 0xFFFFFFFFu;
 constexpr u32 LINK_NIL = 0xFFFFFFFFu;  // end of a destination list (fetch)
@@ -48,7 +66,7 @@ struct Ctrl {
   u32 ev_take;          // promote: where the freed host ids go in the host ring
   u32 ev_host_dropped;  // evict: host-tier drops that made room for a demotion
   u32 live[2];
-  u32 tombstones;
+  u32 max_disp;         // largest distance from its home slot at which a key has ever been placed (0 while below HOP_EXACT)
   u32 pad1;
   // fetch: per-call scalars, double buffered by the call's sequence number so that no launch is needed to clear them:
   // call k uses entry k & 1 and zeroes entry (k + 1) & 1 for the call after it
@@ -68,7 +86,7 @@ struct Ctrl {
   u64 blocks_inserted, blocks_denied;
   u64 blocks_dropped[2];
   u64 blocks_demoted;
-  u64 rebuilds;
+  u64 far_keys;         // keys placed HOP_EXACT or more slots from home so far
   u64 blocks_promoted;
   u64 inflation;        // GDSF clock L: largest priority evicted so far
   u64 blocks_fetched_distinct;   // distinct source blocks read by fetch calls (<= blocks fetched)
@@ -145,85 +163,198 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
   Slot s;
   s.key = ((u64)v.y << 32) | v.x;
   s.id = v.z;
-  s.aux = v.w;
+  s.hop = v.w;
   return s;
 }
+__device__ __forceinline__ u64 wrap_slot(u64 t, u64 slots) { return t >= slots ? t - slots : t; }   // t < 2 * slots
+__device__ __forceinline__ u32 displacement(u64 slot, u64 home, u64 slots) { return (u32)(slot >= home ? slot - home : slot + slots - home); }
 
-// Linear probe for `key`.  Returns the slot index or NO_SLOT; *visited gets the slots examined.
-// The walk is latency bound (each slot is a dependent L2 access) and a warp waits for its slowest lane, so
-// PROBE_WINDOW consecutive slots are loaded at once and then examined in order: a miss at load factor 0.7
-// needs ~6 slots on average with a long tail, which becomes two round trips instead of six or more.
+// Lookup of `key` (see Slot).  One round trip loads the home slot - whose hop word names the slots that matter - and
+// its three neighbours; keys placed further away cost a second round trip for exactly the flagged slots or groups.
+// Split in two so that a caller can put independent work between the loads and their use.  *visited gets the slots
+// compared; the slot index is returned through *slot_out when asked for.
 constexpr int PROBE_WINDOW = 4;
-__device__ __forceinline__ u32 find_slot(const Slot* __restrict__ table, u64 slots, u64 key, u32* visited, u32* id_out) {
-  u64 s = home_slot(key, slots);
-  u32 n = 0;
-  for (u64 i = 0; i < slots; i += PROBE_WINDOW) {
-    uint4 v[PROBE_WINDOW];
-    u64 idx[PROBE_WINDOW];
+struct ProbeWindow { uint4 v[PROBE_WINDOW]; };
+__device__ __forceinline__ void probe_issue(const Store& st, u64 key, ProbeWindow& w) {
+  const u64 h = home_slot(key, st.slots);
 #pragma unroll
-    for (int w = 0; w < PROBE_WINDOW; ++w) {
-      u64 t = s + w;
-      idx[w] = t >= slots ? t - slots : t;
-      v[w] = *reinterpret_cast<const uint4*>(table + idx[w]);
-    }
-#pragma unroll
-    for (int w = 0; w < PROBE_WINDOW; ++w) {
-      const u64 k = ((u64)v[w].y << 32) | v[w].x;
-      ++n;
-      if (k == key) { *visited = n; *id_out = v[w].z; return (u32)idx[w]; }
-      if (k == KEY_EMPTY) { *visited = n; *id_out = NO_ID; return NO_SLOT; }
-    }
-    s += PROBE_WINDOW;
-    if (s >= slots) s -= slots;
-  }
-  *visited = n;
-  *id_out = NO_ID;
-  return NO_SLOT;
+  for (int k = 0; k < PROBE_WINDOW; ++k) w.v[k] = *reinterpret_cast<const uint4*>(st.table + wrap_slot(h + k, st.slots));
 }
 
-// The same probe in two halves, so that a caller can put independent work between the loads of the first window and
-// their use: probe_issue starts the loads, probe_finish examines them and walks on if the run is longer.
-struct ProbeWindow { uint4 v[PROBE_WINDOW]; };
-__device__ __forceinline__ void probe_issue(const Slot* __restrict__ table, u64 slots, u64 key, ProbeWindow& w) {
-  const u64 s = home_slot(key, slots);
+// The near part of a lookup, from the loaded window: the flagged slots up to HOP_EXACT - 1 from home.  Returns the id or
+// NO_ID; *far_bits gets the group / far bits that still have to be followed when the key was not found (0 = it is absent).
+__device__ __forceinline__ u32 probe_near(const Store& st, u64 key, const ProbeWindow& w, u32* compared, u32* slot_out, u32* far_bits) {
+  const u64 h = home_slot(key, st.slots);
+  const u32 bits = w.v[0].w;
+  u32 n = 0;
+  *far_bits = 0;
 #pragma unroll
   for (int k = 0; k < PROBE_WINDOW; ++k) {
-    u64 t = s + k;
-    t = t >= slots ? t - slots : t;
-    w.v[k] = *reinterpret_cast<const uint4*>(table + t);
+    if (!((bits >> k) & 1u)) continue;
+    ++n;
+    if ((((u64)w.v[k].y << 32) | w.v[k].x) == key) {
+      *compared = n;
+      *slot_out = (u32)wrap_slot(h + k, st.slots);
+      return w.v[k].z;
+    }
+  }
+  u32 rest = bits & ((1u << HOP_EXACT) - 1u) & ~((1u << PROBE_WINDOW) - 1u);
+  while (rest) {                                   // the flagged slots beyond the window, four loads in flight at a time
+    uint4 q[PROBE_WINDOW];
+    u32 at[PROBE_WINDOW];
+#pragma unroll
+    for (int k = 0; k < PROBE_WINDOW; ++k) {
+      at[k] = NO_SLOT;
+      if (rest) {
+        const int d = __ffs(rest) - 1;
+        rest &= rest - 1;
+        at[k] = (u32)wrap_slot(h + d, st.slots);
+        q[k] = *reinterpret_cast<const uint4*>(st.table + at[k]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < PROBE_WINDOW; ++k) {
+      if (at[k] == NO_SLOT) continue;
+      ++n;
+      if ((((u64)q[k].y << 32) | q[k].x) == key) {
+        *compared = n;
+        *slot_out = at[k];
+        return q[k].z;
+      }
+    }
+  }
+  *compared = n ? n : 1;
+  *slot_out = NO_SLOT;
+  *far_bits = bits & ~((1u << HOP_EXACT) - 1u);
+  return NO_ID;
+}
+
+// The rare part: a group of HOP_GROUP slots per group bit, and for the far bit every slot from HOP_FAR_FROM to the largest
+// distance ever used.  When a range holds no key of this home, the bit that sent the lookup there is cleared in the home's
+// hop word, so that the next lookup of a key that hashes here is short again.  Only lookups and deletions run beside a
+// lookup, never insertions, and neither can make "no key of this home is left there" false; during an insert's claim
+// phase the keys claimed so far are in the table already and count.
+//
+// Two forms.  probe_far_warp: ALL 32 lanes of a warp call it together; the lanes that have bits to follow are served
+// one after the other, each by the whole warp - one slot per lane, one round trip per 32 slots, no arrays in registers.
+// probe_far_lane: any single thread, four loads in flight; out of line and by value so that it costs its callers
+// nothing but a branch.
+__device__ __forceinline__ void probe_far_warp(const Store& st, u64 key, u32 far_bits, u32* id, u32* slot, u32* compared) {
+  const int lane = threadIdx.x & 31;
+  const u64 h = home_slot(key, st.slots);
+  for (unsigned pending = __ballot_sync(FULL, far_bits != 0); pending; pending &= pending - 1) {
+    const int src = __ffs(pending) - 1;
+    const u64 k0 = __shfl_sync(FULL, key, src), h0 = __shfl_sync(FULL, h, src);
+    const u32 b0 = __shfl_sync(FULL, far_bits, src);
+    u32 found_id = NO_ID, found_slot = NO_SLOT, cmp = 0;
+    const u32 last = (b0 & HOP_FAR) ? *reinterpret_cast<volatile u32*>(&st.ctrl->max_disp) : 0;
+    bool far_has_own = false;
+    // ranges of 32 slots: the flagged groups, then (far bit) HOP_FAR_FROM ... last
+    u32 groups = (b0 >> HOP_EXACT) & ((1u << HOP_GROUPS) - 1u);
+    u32 d0 = HOP_FAR_FROM;
+    while (found_id == NO_ID) {
+      u32 base, heal;
+      if (groups) { const u32 g = (u32)__ffs(groups) - 1; groups &= groups - 1; base = HOP_EXACT + g * HOP_GROUP; heal = 1u << (HOP_EXACT + g); }
+      else if ((b0 & HOP_FAR) && d0 <= last) { base = d0; d0 += 32; heal = 0; }
+      else break;
+      const u32 d = base + lane;
+      const bool in = heal ? true : d <= last;
+      const u32 at = (u32)((h0 + d) % st.slots);
+      uint4 v = make_uint4(0u, 0u, NO_ID, 0u);
+      if (in) v = *reinterpret_cast<const uint4*>(st.table + at);
+      const u64 kk = ((u64)v.y << 32) | v.x;
+      const unsigned hit = __ballot_sync(FULL, in && kk == k0);
+      const unsigned own = __ballot_sync(FULL, in && kk >= 2 && home_slot(kk, st.slots) == h0);
+      cmp += heal ? 32 : (last - base + 1 < 32 ? last - base + 1 : 32);
+      if (hit) {
+        const int l = __ffs(hit) - 1;
+        found_id = __shfl_sync(FULL, v.z, l);
+        found_slot = __shfl_sync(FULL, at, l);
+      } else if (heal) {
+        if (!own && lane == 0) atomicAnd(&st.table[h0].hop, ~heal);
+      } else if (own) {
+        far_has_own = true;
+      }
+    }
+    if (found_id == NO_ID && (b0 & HOP_FAR) && !far_has_own && lane == 0) atomicAnd(&st.table[h0].hop, ~HOP_FAR);
+    if (lane == src) { *id = found_id; *slot = found_slot; *compared += cmp; }
   }
 }
-__device__ __forceinline__ u32 probe_finish(const Slot* __restrict__ table, u64 slots, u64 key, const ProbeWindow& w, u32* visited) {
-  u32 n = 0;
-#pragma unroll
-  for (int k = 0; k < PROBE_WINDOW; ++k) {
-    const u64 kk = ((u64)w.v[k].y << 32) | w.v[k].x;
-    ++n;
-    if (kk == key) { *visited = n; return w.v[k].z; }
-    if (kk == KEY_EMPTY) { *visited = n; return NO_ID; }
-  }
-  u64 s = home_slot(key, slots) + PROBE_WINDOW;
-  if (s >= slots) s -= slots;
-  for (u64 i = PROBE_WINDOW; i < slots; i += PROBE_WINDOW) {
-    uint4 v[PROBE_WINDOW];
-#pragma unroll
-    for (int k = 0; k < PROBE_WINDOW; ++k) {
-      u64 t = s + k;
-      t = t >= slots ? t - slots : t;
-      v[k] = *reinterpret_cast<const uint4*>(table + t);
+__device__ __noinline__ uint4 probe_far_lane(Slot* table, u64 slots, const u32* max_disp, u64 key, u64 h, u32 far_bits) {
+  constexpr int B = 4;
+  u32 compared = 0;
+  u32 groups = (far_bits >> HOP_EXACT) & ((1u << HOP_GROUPS) - 1u);
+  bool far_done = !(far_bits & HOP_FAR);
+  while (groups || !far_done) {
+    u32 d0, len, heal;
+    if (groups) { const u32 g = (u32)__ffs(groups) - 1; groups &= groups - 1; d0 = HOP_EXACT + g * HOP_GROUP; len = HOP_GROUP; heal = 1u << (HOP_EXACT + g); }
+    else {
+      far_done = true;
+      const u32 last = *reinterpret_cast<const volatile u32*>(max_disp);
+      if (last < HOP_FAR_FROM) break;
+      d0 = HOP_FAR_FROM; len = last - HOP_FAR_FROM + 1; heal = HOP_FAR;
     }
+    bool any_of_this_home = false;
+    u64 s = (h + d0) % slots;                          // one division here, none per slot
+    for (u32 d = 0; d < len; d += B) {
+      u64 k[B];
+      const u64 s0 = s;
 #pragma unroll
-    for (int k = 0; k < PROBE_WINDOW; ++k) {
-      const u64 kk = ((u64)v[k].y << 32) | v[k].x;
-      ++n;
-      if (kk == key) { *visited = n; return v[k].z; }
-      if (kk == KEY_EMPTY) { *visited = n; return NO_ID; }
+      for (int x = 0; x < B; ++x) {
+        k[x] = d + x < len ? table[s].key : KEY_EMPTY;
+        s = s + 1 == slots ? 0 : s + 1;
+      }
+#pragma unroll
+      for (int x = 0; x < B; ++x) {
+        if (d + x >= len) break;
+        ++compared;
+        if (k[x] == key) {
+          const u32 at = (u32)((s0 + x) % slots);
+          return make_uint4(table[at].id, at, compared, 0);
+        }
+        if (k[x] >= 2 && home_slot(k[x], slots) == h) any_of_this_home = true;
+      }
     }
-    s += PROBE_WINDOW;
-    if (s >= slots) s -= slots;
+    if (!any_of_this_home) atomicAnd(&table[h].hop, ~heal);
   }
-  *visited = n;
-  return NO_ID;
+  return make_uint4(NO_ID, NO_SLOT, compared, 0);
+}
+
+// The whole lookup for one thread on its own ...
+__device__ __forceinline__ u32 probe_finish(const Store& st, u64 key, const ProbeWindow& w, u32* visited, u32* slot_out = nullptr) {
+  u32 slot, far_bits;
+  u32 id = probe_near(st, key, w, visited, &slot, &far_bits);
+  if (far_bits) {
+    const uint4 r = probe_far_lane(st.table, st.slots, &st.ctrl->max_disp, key, home_slot(key, st.slots), far_bits);
+    id = r.x; slot = r.y; *visited += r.z;
+  }
+  if (slot_out) *slot_out = slot;
+  return id;
+}
+// ... and for the 32 lanes of a warp together (lanes with `active` false take part without a key of their own)
+__device__ __forceinline__ u32 probe_finish_warp(const Store& st, bool active, u64 key, const ProbeWindow& w, u32* visited, u32* slot_out = nullptr) {
+  u32 slot = NO_SLOT, far_bits = 0, id = NO_ID;
+  *visited = 0;
+  if (active) id = probe_near(st, key, w, visited, &slot, &far_bits);
+  if (__any_sync(FULL, far_bits != 0)) probe_far_warp(st, key, far_bits, &id, &slot, visited);
+  if (slot_out) *slot_out = slot;
+  return id;
+}
+
+// slot of `key`, or NO_SLOT
+__device__ __forceinline__ u32 find_slot(const Store& st, u64 key, u32* visited, u32* id_out) {
+  ProbeWindow w;
+  probe_issue(st, key, w);
+  u32 slot;
+  *id_out = probe_finish(st, key, w, visited, &slot);
+  return slot;
+}
+__device__ __forceinline__ u32 find_slot_warp(const Store& st, bool active, u64 key, u32* visited, u32* id_out) {
+  ProbeWindow w;
+  if (active) probe_issue(st, key, w);
+  u32 slot;
+  *id_out = probe_finish_warp(st, active, key, w, visited, &slot);
+  return slot;
 }
 
 __device__ __forceinline__ int tier_of(const Store& st, u32 id) { return id < st.n[0] ? 0 : 1; }

@@ -1,4 +1,4 @@
-// Eviction of unreferenced leaves (LRU or GDSF order), demotion to the host tier, table rebuild.
+// Eviction of unreferenced leaves (LRU or GDSF order), demotion to the host tier.
 // (Paper Section 1: blocks of finished requests are evicted least-recently-used first; Section 4.1
 // "Access pattern-aware eviction policy": owned tensors are flushed to slower tiers, not dropped.)
 //
@@ -59,7 +59,7 @@ __device__ __forceinline__ void mark_blocked_walk(const Store& st, unsigned char
   bool climbing = false;
   for (u32 step = 0; step < 65536; ++step) {
     u32 visited, pid;
-    if (find_slot(st.table, st.slots, pk, &visited, &pid) == NO_SLOT || pid == NO_ID) break;
+    if (find_slot(st, pk, &visited, &pid) == NO_SLOT || pid == NO_ID) break;
     if (pid >= st.n[0]) {                                   // host-tier ancestor
       if (*reinterpret_cast<volatile unsigned char*>(&blocked[pid])) break;
       blocked[pid] = 1;
@@ -110,7 +110,6 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
 
   // ---- what is wanted; ring positions are read now, before anything in this launch changes them ----------------------
   const u32 head0 = c->ring[0].head, count0 = c->ring[0].count, head1 = c->ring[1].head, count1 = c->ring[1].count;
-  const u32 tomb0 = c->tombstones;
   const u32 host_dropped = c->ev_host_dropped;
   u32 n = a.n;
   if (a.want_free >= 0) {                      // reserve form: every CTA sums the list for itself
@@ -269,11 +268,14 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
       if (bar.ok) {
         const Key2* sorted = a.buf[cur];
         if (a.mode == EV_DEMOTE) {
-          for (u32 i = blockIdx.x * EV_THREADS + threadIdx.x; i < take; i += G * EV_THREADS) {
-            const u32 old_id = (u32)(sorted[i].lo & 0xFFFFFFFFu);
-            const u32 new_id = (u32)st.ring_ids[1][(u32)(((u64)head1 + i) % st.n[1])];
+          for (u32 i0 = blockIdx.x * EV_THREADS + (threadIdx.x & ~31u); i0 < take; i0 += G * EV_THREADS) {   // whole warps
+            const u32 i = i0 + (threadIdx.x & 31u);
+            const bool on = i < take;
+            const u32 old_id = on ? (u32)(sorted[i].lo & 0xFFFFFFFFu) : 0;
             u32 visited, sid;
-            const u32 s = find_slot(st.table, st.slots, st.m_key[old_id], &visited, &sid);
+            const u32 s = find_slot_warp(st, on, on ? st.m_key[old_id] : 0, &visited, &sid);
+            if (!on) continue;
+            const u32 new_id = (u32)st.ring_ids[1][(u32)(((u64)head1 + i) % st.n[1])];
             if (s != NO_SLOT) st.table[s].id = new_id;
             st.m_key[new_id] = st.m_key[old_id];
             st.m_parent[new_id] = st.m_parent[old_id];
@@ -290,14 +292,20 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
         } else {
           int* victims = a.mode == EV_DROP ? a.victims : a.room;
           const u32 cap = st.n[tier], head = tier ? head1 : head0, count = tier ? count1 : count0;
-          for (u32 i = blockIdx.x * EV_THREADS + threadIdx.x; i < take; i += G * EV_THREADS) {
-            const u32 id = (u32)(sorted[i].lo & 0xFFFFFFFFu);
+          for (u32 i0 = blockIdx.x * EV_THREADS + (threadIdx.x & ~31u); i0 < take; i0 += G * EV_THREADS) {   // whole warps
+            const u32 i = i0 + (threadIdx.x & 31u);
+            const bool on = i < take;
+            const u32 id = on ? (u32)(sorted[i].lo & 0xFFFFFFFFu) : 0;
             u32 visited, sid;
-            const u32 s = find_slot(st.table, st.slots, st.m_key[id], &visited, &sid);
-            if (s != NO_SLOT) {
+            const u64 key = on ? st.m_key[id] : 0;
+            const u32 s = find_slot_warp(st, on, key, &visited, &sid);
+            if (!on) continue;
+            if (s != NO_SLOT) {                     // the slot is empty again; a group or far bit stays (lookups clear those)
+              const u64 h = home_slot(key, st.slots);
+              const u32 d = displacement(s, h, st.slots);
               st.table[s].id = NO_ID;
-              st.table[s].aux = NO_ID;
-              st.table[s].key = KEY_TOMB;
+              st.table[s].key = KEY_EMPTY;
+              if (d < HOP_EXACT) atomicAnd(&st.table[h].hop, ~(1u << d));
             }
             st.m_key[id] = 0;
             st.ring_ids[tier][(u32)(((u64)head + count + i) % cap)] = (int)id;
@@ -330,7 +338,6 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
     } else {
       c->ring[tier].count = (tier ? count1 : count0) + take;
       c->live[tier] -= take;
-      c->tombstones = tomb0 + take;
       c->blocks_dropped[tier] += take;
       if (a.mode == EV_DROP) { if (a.n_evicted) { a.n_evicted[0] = (int)take; a.n_evicted[1] = 0; } }
       else c->ev_host_dropped = take;
@@ -338,34 +345,9 @@ __global__ void __launch_bounds__(EV_THREADS) evict_kernel(Store st, EvictArgs a
   }
 }
 
-// ---- table maintenance ------------------------------------------------------------------------------------
-// Rebuild in place, by every CTA of a cooperative launch: the table is moved aside (stash), cleared, and its live
-// entries are put back, which reclaims the deleted markers.  Two barriers; the caller resets the marker count.
-__device__ __forceinline__ void table_rebuild_coop(const Store& st, Slot* __restrict__ stash, GridBarrier& bar) {
-  const u64 stride = (u64)gridDim.x * blockDim.x;
-  for (u64 s = (u64)blockIdx.x * blockDim.x + threadIdx.x; s < st.slots; s += stride) {
-    uint4* p = reinterpret_cast<uint4*>(st.table + s);
-    *reinterpret_cast<uint4*>(stash + s) = *p;
-    *p = make_uint4(0u, 0u, NO_ID, NO_ID);
-  }
-  if (!bar.sync(st)) return;
-  for (u64 s = (u64)blockIdx.x * blockDim.x + threadIdx.x; s < st.slots; s += stride) {
-    const Slot v = load_slot(stash + s);
-    if (v.key < 2 || v.id == NO_ID) continue;
-    u64 t = home_slot(v.key, st.slots);
-    bool placed = false;
-    for (u64 i = 0; i < st.slots; ++i) {
-      if (atomicCAS(&st.table[t].key, KEY_EMPTY, v.key) == KEY_EMPTY) { st.table[t].id = v.id; placed = true; break; }
-      t = (t + 1 == st.slots) ? 0 : t + 1;
-    }
-    if (!placed) raise(st, S_TABLE_FULL);
-  }
-  bar.sync(st);
-}
-
 __global__ void __launch_bounds__(256) table_clear_kernel(Slot* __restrict__ table, u64 slots) {
   for (u64 s = (u64)blockIdx.x * blockDim.x + threadIdx.x; s < slots; s += (u64)gridDim.x * blockDim.x) {
-    uint4 v = make_uint4(0u, 0u, NO_ID, NO_ID);
+    uint4 v = make_uint4(0u, 0u, NO_ID, 0u);
     *reinterpret_cast<uint4*>(table + s) = v;
   }
 }
@@ -392,8 +374,8 @@ __global__ void ctrl_init_kernel(Store st, u64* __restrict__ progress, int n_pro
 
 // counters for a caller that does not want to block: written by the device to any device-accessible address
 struct StatsOut {
-  u64 epoch, live[2], free_blocks[2], tombstones, query_blocks, probes_issued, slots_visited, blocks_matched, blocks_fetched[2],
-      blocks_inserted, blocks_denied, blocks_dropped[2], blocks_demoted, rebuilds, blocks_promoted, gdsf_clock, blocks_fetched_distinct;
+  u64 epoch, live[2], free_blocks[2], max_displacement, query_blocks, probes_issued, slots_visited, blocks_matched, blocks_fetched[2],
+      blocks_inserted, blocks_denied, blocks_dropped[2], blocks_demoted, far_keys, blocks_promoted, gdsf_clock, blocks_fetched_distinct;
 };
 __global__ void stats_kernel(Store st, u64 epoch, StatsOut* __restrict__ out) {
   const Ctrl* c = st.ctrl;
@@ -403,14 +385,14 @@ __global__ void stats_kernel(Store st, u64 epoch, StatsOut* __restrict__ out) {
     o.live[t] = c->live[t]; o.free_blocks[t] = c->ring[t].count;
     o.blocks_fetched[t] = c->blocks_fetched[t]; o.blocks_dropped[t] = c->blocks_dropped[t];
   }
-  o.tombstones = c->tombstones;
+  o.max_displacement = c->max_disp;
   o.query_blocks = c->query_blocks; o.probes_issued = c->probes_issued; o.slots_visited = c->slots_visited; o.blocks_matched = c->blocks_matched;
   for (int i = 0; i < LOOKUP_STRIPES; ++i) {
     o.query_blocks += c->lookup_stripes[i][0]; o.probes_issued += c->lookup_stripes[i][1];
     o.slots_visited += c->lookup_stripes[i][2]; o.blocks_matched += c->lookup_stripes[i][3];
   }
   o.blocks_inserted = c->blocks_inserted; o.blocks_denied = c->blocks_denied; o.blocks_demoted = c->blocks_demoted;
-  o.rebuilds = c->rebuilds; o.blocks_promoted = c->blocks_promoted; o.gdsf_clock = c->inflation;
+  o.far_keys = c->far_keys; o.blocks_promoted = c->blocks_promoted; o.gdsf_clock = c->inflation;
   o.blocks_fetched_distinct = c->blocks_fetched_distinct;
   *out = o;
 }

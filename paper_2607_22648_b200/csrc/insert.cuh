@@ -4,18 +4,17 @@
 // The batch must behave as if requests were inserted one after the other in index order.  All the
 // metadata work of a call runs in ONE cooperative kernel whose phases are separated by grid-wide
 // barriers (elements e = (request r, block j), R*max_blocks of them):
-//   rebuild : only when deleted table markers have piled up: move the table aside, clear it, put the
-//             live entries back.
 //   hash    : chained block keys (content hashes first, by one thread per block, when requests are few
 //             and long); serial along a request
-//   claim   : find the key of e in the table or claim an empty slot for it (atomicCAS on the key);
-//             every element that lands on a slot claimed in this call lowers slot.aux to its request
-//             index (atomicMin), so the lowest request presenting a new prefix becomes its creator.
+//   claim   : find the key of e in the table or claim the first empty slot at or after its home slot
+//             (atomicCAS on the key); every element that lands on a slot claimed in this call lowers
+//             slot.id to ID_PENDING | its request index (atomicMin), so the lowest request presenting a
+//             new prefix becomes its creator.
 //   count   : flag(e) = "e creates a node"; sums per tile of 1024 elements.
 //   assign  : every CTA derives the allocation plan from the tile sums (grants = min(new nodes, free HBM
 //             blocks)); rank(e) among creators in (r, j) order; rank < grants gets ring[head + rank],
-//             writes the slot value, the node's metadata and a copy descriptor; the others delete
-//             their claim.
+//             writes the slot value, flags the slot in its home slot's hop word, writes the node's
+//             metadata and a copy descriptor; the others empty their slot again.
 //   finish  : every element reads its slot's block id (or -1) and refreshes the LRU stamp.
 // Ranking creators in (r, j) order and granting the first `free` of them equals the sequential rule:
 // a denied node's descendants always rank higher, so denials are prefix-closed per request.
@@ -32,7 +31,7 @@ __device__ __forceinline__ u32 creator_flag(const Store& st, const u32* __restri
   const u32 s = eslot[e];
   if (s == NO_SLOT) return 0;
   const Slot v = load_slot(st.table + s);
-  return (v.id == NO_ID && v.aux == (u32)(e / max_blocks)) ? 1u : 0u;
+  return v.id == (ID_PENDING | (u32)(e / max_blocks)) ? 1u : 0u;
 }
 
 // block-wide inclusive scan of one value per thread (INS_THREADS threads); returns inclusive sum, total in *total
@@ -53,36 +52,45 @@ __device__ __forceinline__ u32 block_scan_incl(u32 x, u32* warp_sums, u32* total
   return incl;
 }
 
-// find `key` or claim an empty slot for it; the lowest request index presenting a key claimed in this call owns it.
-// The probe run is read PROBE_WINDOW slots at a time (one round trip instead of four dependent ones).  Values read
-// early stay usable: during the claim phase a slot only ever changes from empty to a key, and an empty slot is never
-// passed over, it is claimed with a compare-and-swap whose result says what the slot really holds.
-__device__ __forceinline__ u32 claim_slot(const Store& st, u64 key, u32 r) {
+// Find `key` or claim a slot for it; the lowest request index presenting a key claimed in this call owns it.
+// First the lookup proper (home slot, flagged slots): a key stored by an earlier call is found there and nowhere else.
+// A new key then takes the first empty slot at or after its home slot.  The walk reads PROBE_WINDOW slots at a time
+// and compares every key it passes, because another element of this call may be claiming the same key at the same
+// time: all of them walk the same slots in the same order, an empty slot is never passed over but claimed with a
+// compare-and-swap whose result says what the slot really holds, and during this phase a slot only ever changes from
+// empty to a key - so the first claim is seen by everyone who comes later.  (Keys claimed in this call are flagged in
+// their home slots only when they are granted a block, after the phase.)
+// Called by all 32 lanes of a warp together (lanes without an element pass active = false).
+__device__ __forceinline__ u32 claim_slot(const Store& st, bool active, u64 key, u32 r) {
+  ProbeWindow w;
+  if (active) probe_issue(st, key, w);
+  u32 visited, got;
+  const u32 id = probe_finish_warp(st, active, key, w, &visited, &got);
+  if (!active) return NO_SLOT;
+  if (id != NO_ID) return got;                       // an existing node
+  got = NO_SLOT;
   u64 s = home_slot(key, st.slots);
-  u32 got = NO_SLOT;
   for (u64 i = 0; i < st.slots && got == NO_SLOT; i += PROBE_WINDOW) {
     u64 k[PROBE_WINDOW], idx[PROBE_WINDOW];
 #pragma unroll
-    for (int w = 0; w < PROBE_WINDOW; ++w) {
-      const u64 t = s + w;
-      idx[w] = t >= st.slots ? t - st.slots : t;
-      k[w] = *reinterpret_cast<volatile u64*>(&st.table[idx[w]].key);
+    for (int x = 0; x < PROBE_WINDOW; ++x) {
+      idx[x] = wrap_slot(s + x, st.slots);
+      k[x] = i == 0 ? (((u64)w.v[x].y << 32) | w.v[x].x) : *reinterpret_cast<volatile u64*>(&st.table[idx[x]].key);
     }
 #pragma unroll
-    for (int w = 0; w < PROBE_WINDOW; ++w) {
+    for (int x = 0; x < PROBE_WINDOW; ++x) {
       if (got != NO_SLOT) break;
-      u64 kk = k[w];
+      u64 kk = k[x];
       if (kk == KEY_EMPTY) {
-        kk = atomicCAS(&st.table[idx[w]].key, KEY_EMPTY, key);
+        kk = atomicCAS(&st.table[idx[x]].key, KEY_EMPTY, key);
         if (kk == KEY_EMPTY) kk = key;                 // claimed
       }
-      if (kk == key) got = (u32)idx[w];
+      if (kk == key) got = (u32)idx[x];
     }
-    s += PROBE_WINDOW;
-    if (s >= st.slots) s -= st.slots;
+    s = wrap_slot(s + PROBE_WINDOW, st.slots);
   }
   if (got == NO_SLOT) { raise(st, S_TABLE_FULL); return got; }
-  if (*reinterpret_cast<volatile u32*>(&st.table[got].id) == NO_ID) atomicMin(&st.table[got].aux, r);
+  atomicMin(&st.table[got].id, ID_PENDING | r);        // NO_ID or another request's mark: the lowest request stays
   return got;
 }
 
@@ -102,8 +110,6 @@ struct InsertArgs {
   int2* desc;               // out: copy descriptors {pool block, cache block}, ctrl->n_pairs of them
   int* ids_out;
   int* new_blocks;
-  Slot* stash;
-  u32 rebuild_threshold;
   u32 launch_seq;
 };
 
@@ -118,14 +124,12 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
   const long long total = (long long)a.R * a.max_blocks;
   const int max_blocks = a.max_blocks;
   // plan inputs, read before anything in this launch changes them
-  const u32 head0 = c->ring[0].head, count0 = c->ring[0].count, tomb0 = c->tombstones;
+  const u32 head0 = c->ring[0].head, count0 = c->ring[0].count;
   const u64 inflation = st.policy ? c->inflation : 0;
   const long long gthreads = (long long)gridDim.x * INS_THREADS;
   const long long gtid = (long long)blockIdx.x * INS_THREADS + threadIdx.x;
 
   PHASE_MARK(st, 0);
-  const bool rebuild = tomb0 > a.rebuild_threshold;
-  if (rebuild) table_rebuild_coop(st, a.stash, bar);
   PHASE_MARK(st, 1);
 
   // ---- hash + claim ----------------------------------------------------------------------------------------------------
@@ -175,9 +179,11 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
   bar.sync(st);
   PHASE_MARK(st, 3);
   // the chain is serial per request, the claims are not: one element per thread, so that the probe latencies overlap
-  for (long long e = gtid; e < total && bar.ok; e += gthreads) {
-    const u64 key = a.keys[e];
-    a.eslot[e] = key ? claim_slot(st, key, (u32)(e / max_blocks)) : NO_SLOT;
+  for (long long e0 = gtid - lane; e0 < total && bar.ok; e0 += gthreads) {        // whole warps: claim_slot wants all lanes
+    const long long e = e0 + lane;
+    const u64 key = e < total ? a.keys[e] : 0;
+    const u32 s = claim_slot(st, key != 0, key, (u32)(e / max_blocks));
+    if (e < total) a.eslot[e] = s;
   }
   bar.sync(st);
   PHASE_MARK(st, 4);
@@ -203,7 +209,6 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
   }
   const u32 granted = total_new < count0 ? total_new : count0;
   if (blockIdx.x == 0 && threadIdx.x == 0 && bar.ok) {
-    if (rebuild) c->rebuilds += 1;
     c->ins_total_new = total_new;
     c->ins_granted = granted;
     c->ins_base = head0;
@@ -213,7 +218,6 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     c->n_pairs = granted;
     c->blocks_inserted += granted;
     c->blocks_denied += total_new - granted;
-    c->tombstones = (rebuild ? 0 : tomb0) + (total_new - granted);
     if (granted < total_new) atomicOr(&c->status, S_NOSPACE);
   }
   for (long long t = blockIdx.x; t < n_tiles && bar.ok; t += gridDim.x) {
@@ -230,9 +234,9 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     if (!f) continue;
     const u32 rank = before + incl - 1;
     Slot* slot = st.table + a.eslot[e];
-    if (rank >= granted) {                       // denied: withdraw the claim
-      slot->aux = NO_ID;
-      slot->key = KEY_TOMB;
+    if (rank >= granted) {                       // denied: the slot is empty again (nobody walks the table in this phase)
+      slot->id = NO_ID;
+      slot->key = KEY_EMPTY;
       continue;
     }
     const u32 id = (u32)st.ring_ids[0][(u32)(((u64)head0 + rank) % st.n[0])];
@@ -243,8 +247,13 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     st.m_freq[id] = 0;
     st.m_ref[id] = 0;
     st.m_depth[id] = (u32)j;
-    slot->aux = NO_ID;
     slot->id = id;
+    {                                            // make the key findable: flag its slot in the home slot's hop word
+      const u64 h = home_slot(a.keys[e], st.slots);
+      const u32 d = displacement(a.eslot[e], h, st.slots);
+      atomicOr(&st.table[h].hop, hop_bit(d));
+      if (d >= HOP_EXACT) { atomicMax(&c->max_disp, d); atomicAdd(&c->far_keys, 1ull); }
+    }
     int2 d = make_int2((int)id, 0);
     if (a.bt) {
       const int cb = a.bt[e];
@@ -266,7 +275,7 @@ __global__ void __launch_bounds__(INS_THREADS) insert_kernel(Store st, InsertArg
     int out = -1;
     if (s != NO_SLOT) {
       const u32 id = st.table[s].id;
-      if (id != NO_ID) { out = (int)id; touch_block(st, id, a.epoch, inflation, 1); }
+      if (id < ID_PENDING) { out = (int)id; touch_block(st, id, a.epoch, inflation, 1); }
     }
     a.ids_out[e] = out;
   }

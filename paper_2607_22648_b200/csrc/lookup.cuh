@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(256) hash_kernel(Store st, const int* __restri
 }
 
 template <int L>
-__global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __restrict__ tokens,
+__global__ void __launch_bounds__(256, 4) lookup_kernel(Store st, const int* __restrict__ tokens,
                                                      const long long* __restrict__ offsets, int R, int max_blocks,
                                                      u32 flags, u64 epoch, int* __restrict__ matched,
                                                      int* __restrict__ ids_out, FetchLink fl, u64* __restrict__ keys_out,
@@ -162,17 +162,19 @@ __global__ void __launch_bounds__(256) lookup_kernel(Store st, const int* __rest
     // one probe per distinct key in the warp
     u32 id = NO_ID;
     const unsigned act = __ballot_sync(FULL, active);
+    unsigned peers = 0;
+    int leader = lane;
     if (active) {
-      const unsigned peers = __match_any_sync(act, key);
-      const int leader = __ffs(peers) - 1;
-      if (lane == leader) {
-        u32 visited;
-        find_slot(st.table, st.slots, key, &visited, &id);
-        my_probes += 1;
-        my_visited += visited;
-      }
-      id = __shfl_sync(peers, id, leader);
+      peers = __match_any_sync(act, key);
+      leader = __ffs(peers) - 1;
     }
+    {
+      const bool probing = active && lane == leader;
+      u32 visited;
+      find_slot_warp(st, probing, key, &visited, &id);          // all lanes: the rare long way is walked by the whole warp
+      if (probing) { my_probes += 1; my_visited += visited; }
+    }
+    if (active) id = __shfl_sync(peers, id, leader);
     // first miss inside each sub-warp
     const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
     const unsigned mine = (found >> (sub * L)) & SUBMASK;
@@ -295,7 +297,7 @@ __device__ __forceinline__ int chain_probe_request(const Store& st, u64* crow, i
     const int j = base + lane;
     const bool active = j < nblk;
     ProbeWindow w;
-    if (active) probe_issue(st.table, st.slots, key, w);          // loads in flight ...
+    if (active) probe_issue(st, key, w);          // loads in flight ...
     u64 next_key = 0;
     if (base + 32 < nblk) {                                       // ... while the next chunk is chained
       const u64 cn = c_next;
@@ -307,11 +309,10 @@ __device__ __forceinline__ int chain_probe_request(const Store& st, u64* crow, i
     if (active) crow[j] = key;                // the content hashes of this chunk and the next are in registers by now
     n_hashed = nblk < base + 32 ? nblk : base + 32;
     u32 id = NO_ID;
-    if (active) {
+    {
       u32 visited;
-      id = probe_finish(st.table, st.slots, key, w, &visited);
-      probes += 1;
-      visited_sum += visited;
+      id = probe_finish_warp(st, active, key, w, &visited);       // all lanes: the rare long way is walked by the whole warp
+      if (active) { probes += 1; visited_sum += visited; }
     }
     const unsigned found = __ballot_sync(FULL, active && id != NO_ID);
     const int nf = (found == FULL) ? 32 : (__ffs(~found) - 1);

@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(INS_THREADS) promote_assign_kernel(Store st, c
   const u32 new_id = (u32)st.ring_ids[0][(u32)(((u64)c->ins_base + rank) % st.n[0])];
   st.ring_ids[1][(u32)(((u64)c->ev_take + rank) % st.n[1])] = (int)old_id;
   u32 visited, sid;
-  const u32 s = find_slot(st.table, st.slots, st.m_key[old_id], &visited, &sid);
+  const u32 s = find_slot(st, st.m_key[old_id], &visited, &sid);
   if (s != NO_SLOT) st.table[s].id = new_id;
   st.m_key[new_id] = st.m_key[old_id];
   st.m_parent[new_id] = st.m_parent[old_id];

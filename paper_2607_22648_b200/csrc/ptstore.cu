@@ -23,7 +23,7 @@ constexpr u64 ALIGN = 256;
 inline u64 align_up(u64 x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {            // byte offsets into the workspace
-  u64 table[2], m_key, m_parent, m_last, m_freq, m_ref, m_depth, m_flight, ring[2], ctrl, blocked, sort[2], hist, tile_stats, room, desc,
+  u64 table, m_key, m_parent, m_last, m_freq, m_ref, m_depth, m_flight, ring[2], ctrl, blocked, sort[2], hist, tile_stats, room, desc,
       keys, eslot, cta_sums, prefix, promo_first, promo_cnt, heads, links, desc_tier, desc_host, progress, total;
 };
 
@@ -49,8 +49,7 @@ Layout make_layout(const ptstore_config_t* c) {
   const u64 N = (u64)c->hbm_blocks + c->host_blocks, M = c->max_batch_blocks, S = effective_slots(c);
   u64 o = 0;
   auto take = [&](u64 bytes) { u64 at = o; o = align_up(o + (bytes ? bytes : 1)); return at; };
-  L.table[0] = take(S * sizeof(Slot));
-  L.table[1] = take(S * sizeof(Slot));
+  L.table = take(S * sizeof(Slot));
   L.m_key = take(N * 8); L.m_parent = take(N * 8); L.m_last = take(N * 8);
   L.m_freq = take(N * 4); L.m_ref = take(N * 4); L.m_depth = take(N * 4); L.m_flight = take(N * 4);
   L.ring[0] = take((u64)c->hbm_blocks * 4); L.ring[1] = take((u64)c->host_blocks * 4);
@@ -86,7 +85,6 @@ struct ptstore {
   ptstore_config_t cfg;
   Layout lay;
   Store st;
-  Slot* stash;           // second table-sized buffer used by the in-place rebuild
   unsigned char* blocked;
   Key2* sort_buf[2];
   u32* hist;
@@ -333,9 +331,6 @@ int launch_copy(ptstore* h, const Paged& pc, bool host_side_possible, cudaStream
   return PTSTORE_OK;
 }
 
-// deleted markers are reclaimed at the start of an insert once they exceed 1/8 of the table (device-side decision)
-inline u32 rebuild_threshold(const ptstore* h) { return (u32)(h->st.slots / 8); }
-
 // make `s` wait for a demotion copy left running on the side stream
 int join_tier(ptstore* h, cudaStream_t s) {
   if (!h->tier_pending) return PTSTORE_OK;
@@ -545,9 +540,8 @@ int ptstore_create(const ptstore_config_t* cfg, ptstore_t** out, ptstore_stream_
   h->coop_grid = sms < (int)MAX_COOP_GRID ? sms : (int)MAX_COOP_GRID;
   h->wait_limit = BULK_POLL_LIMIT;
   unsigned char* w = static_cast<unsigned char*>(cfg->workspace);
-  h->stash = reinterpret_cast<Slot*>(w + lay.table[1]);
   Store& st = h->st;
-  st.table = reinterpret_cast<Slot*>(w + lay.table[0]);
+  st.table = reinterpret_cast<Slot*>(w + lay.table);
   st.slots = effective_slots(cfg);
   st.m_key = reinterpret_cast<u64*>(w + lay.m_key);
   st.m_parent = reinterpret_cast<u64*>(w + lay.m_parent);
@@ -719,8 +713,6 @@ static int insert_entry(ptstore_t* h, const int32_t* tokens, const int64_t* offs
   a.epoch = h->epoch;
   a.desc = h->desc;
   a.ids_out = block_ids; a.new_blocks = new_blocks;
-  a.stash = h->stash;
-  a.rebuild_threshold = rebuild_threshold(h);
   // CTAs: enough for one element per thread and for one sub-warp per request, at most one per SM
   const long long by_elems = (total + INS_THREADS - 1) / INS_THREADS;
   const long long by_reqs = ((long long)R * lanes + INS_THREADS - 1) / INS_THREADS;
@@ -868,7 +860,7 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
     out->blocks_fetched[t] = c.blocks_fetched[t];
     out->blocks_dropped[t] = c.blocks_dropped[t];
   }
-  out->tombstones = c.tombstones;
+  out->max_displacement = c.max_disp;
   out->query_blocks = c.query_blocks;
   out->probes_issued = c.probes_issued;
   out->slots_visited = c.slots_visited;
@@ -882,7 +874,7 @@ int ptstore_stats(ptstore_t* h, ptstore_stream_t stream, ptstore_stats_t* out) {
   out->blocks_inserted = c.blocks_inserted;
   out->blocks_denied = c.blocks_denied;
   out->blocks_demoted = c.blocks_demoted;
-  out->rebuilds = c.rebuilds;
+  out->far_keys = c.far_keys;
   out->blocks_promoted = c.blocks_promoted;
   out->gdsf_clock = c.inflation;
   out->blocks_fetched_distinct = c.blocks_fetched_distinct;

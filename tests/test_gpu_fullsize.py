@@ -180,7 +180,7 @@ def test_medium_serving_loops_where_cooperative_kernels_span_several_ctas(host, 
     meeting at grid barriers), insert metadata over 2,500-20,000 elements (3-20 CTAs), long prompts (one CTA per request)
     and thousands of short ones (sub-warps, lists linked inside the chunk loop; "long8": 12 prompts and no host tier, so the
     fused call is the single lookup + gather launch); two thirds of the steps use the fused calls,
-    the rest the separate ones with promotion and asynchronous demotion; table rebuilds happen every few steps."""
+    the rest the separate ones with promotion and asynchronous demotion."""
     from tests.serving import LockstepServing
     if shape.startswith("long"):
         bt = int(shape[4:])
@@ -203,7 +203,7 @@ def test_medium_serving_loops_where_cooperative_kernels_span_several_ctas(host, 
         evicting += r["evicted"] is not None
     s = srv.check_counts()
     assert srv.check_pool(16) > 0
-    assert evicting > steps // 2 and s.rebuilds > 0
+    assert evicting > steps // 2
     if shape.startswith("long"):
         assert srv.g.resumed_inserts() == len([k for k in range(steps) if k % 3 != 2])
     srv.close()
