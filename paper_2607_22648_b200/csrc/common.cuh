@@ -174,54 +174,44 @@ __device__ __forceinline__ u32 displacement(u64 slot, u64 home, u64 slots) { ret
 // Split in two so that a caller can put independent work between the loads and their use.  *visited gets the slots
 // compared; the slot index is returned through *slot_out when asked for.
 constexpr int PROBE_WINDOW = 4;
-struct ProbeWindow { uint4 v[PROBE_WINDOW]; };
+struct ProbeWindow { uint4 v0, v1, v2, v3; };       // named members: an indexed array ended up in local memory
 __device__ __forceinline__ void probe_issue(const Store& st, u64 key, ProbeWindow& w) {
   const u64 h = home_slot(key, st.slots);
-#pragma unroll
-  for (int k = 0; k < PROBE_WINDOW; ++k) w.v[k] = *reinterpret_cast<const uint4*>(st.table + wrap_slot(h + k, st.slots));
+  w.v0 = *reinterpret_cast<const uint4*>(st.table + h);
+  w.v1 = *reinterpret_cast<const uint4*>(st.table + wrap_slot(h + 1, st.slots));
+  w.v2 = *reinterpret_cast<const uint4*>(st.table + wrap_slot(h + 2, st.slots));
+  w.v3 = *reinterpret_cast<const uint4*>(st.table + wrap_slot(h + 3, st.slots));
 }
+__device__ __forceinline__ u64 slot_key(const uint4& v) { return ((u64)v.y << 32) | v.x; }
 
 // The near part of a lookup, from the loaded window: the flagged slots up to HOP_EXACT - 1 from home.  Returns the id or
 // NO_ID; *far_bits gets the group / far bits that still have to be followed when the key was not found (0 = it is absent).
 __device__ __forceinline__ u32 probe_near(const Store& st, u64 key, const ProbeWindow& w, u32* compared, u32* slot_out, u32* far_bits) {
   const u64 h = home_slot(key, st.slots);
-  const u32 bits = w.v[0].w;
+  const u32 bits = w.v0.w;
   u32 n = 0;
   *far_bits = 0;
-#pragma unroll
-  for (int k = 0; k < PROBE_WINDOW; ++k) {
-    if (!((bits >> k) & 1u)) continue;
-    ++n;
-    if ((((u64)w.v[k].y << 32) | w.v[k].x) == key) {
-      *compared = n;
-      *slot_out = (u32)wrap_slot(h + k, st.slots);
-      return w.v[k].z;
-    }
-  }
+  if (bits & 1u) { ++n; if (slot_key(w.v0) == key) { *compared = n; *slot_out = (u32)h; return w.v0.z; } }
+  if (bits & 2u) { ++n; if (slot_key(w.v1) == key) { *compared = n; *slot_out = (u32)wrap_slot(h + 1, st.slots); return w.v1.z; } }
+  if (bits & 4u) { ++n; if (slot_key(w.v2) == key) { *compared = n; *slot_out = (u32)wrap_slot(h + 2, st.slots); return w.v2.z; } }
+  if (bits & 8u) { ++n; if (slot_key(w.v3) == key) { *compared = n; *slot_out = (u32)wrap_slot(h + 3, st.slots); return w.v3.z; } }
   u32 rest = bits & ((1u << HOP_EXACT) - 1u) & ~((1u << PROBE_WINDOW) - 1u);
-  while (rest) {                                   // the flagged slots beyond the window, four loads in flight at a time
-    uint4 q[PROBE_WINDOW];
-    u32 at[PROBE_WINDOW];
-#pragma unroll
-    for (int k = 0; k < PROBE_WINDOW; ++k) {
-      at[k] = NO_SLOT;
-      if (rest) {
-        const int d = __ffs(rest) - 1;
-        rest &= rest - 1;
-        at[k] = (u32)wrap_slot(h + d, st.slots);
-        q[k] = *reinterpret_cast<const uint4*>(st.table + at[k]);
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < PROBE_WINDOW; ++k) {
-      if (at[k] == NO_SLOT) continue;
-      ++n;
-      if ((((u64)q[k].y << 32) | q[k].x) == key) {
-        *compared = n;
-        *slot_out = at[k];
-        return q[k].z;
-      }
-    }
+  while (rest) {                                   // the flagged slots beyond the window, up to four loads in flight
+    const int d0 = __ffs(rest) - 1; rest &= rest - 1;
+    const int d1 = rest ? __ffs(rest) - 1 : d0; rest &= rest - 1;
+    const int d2 = rest ? __ffs(rest) - 1 : d0; rest &= rest - 1;
+    const int d3 = rest ? __ffs(rest) - 1 : d0; rest &= rest - 1;
+    const u32 a0 = (u32)wrap_slot(h + d0, st.slots), a1 = (u32)wrap_slot(h + d1, st.slots);
+    const u32 a2 = (u32)wrap_slot(h + d2, st.slots), a3 = (u32)wrap_slot(h + d3, st.slots);
+    const uint4 q0 = *reinterpret_cast<const uint4*>(st.table + a0);
+    const uint4 q1 = *reinterpret_cast<const uint4*>(st.table + a1);      // a repeat of the first slot when fewer are flagged
+    const uint4 q2 = *reinterpret_cast<const uint4*>(st.table + a2);
+    const uint4 q3 = *reinterpret_cast<const uint4*>(st.table + a3);
+    n += 1u + (d1 != d0) + (d2 != d0) + (d3 != d0);
+    if ((((u64)q0.y << 32) | q0.x) == key) { *compared = n; *slot_out = a0; return q0.z; }
+    if ((((u64)q1.y << 32) | q1.x) == key) { *compared = n; *slot_out = a1; return q1.z; }
+    if ((((u64)q2.y << 32) | q2.x) == key) { *compared = n; *slot_out = a2; return q2.z; }
+    if ((((u64)q3.y << 32) | q3.x) == key) { *compared = n; *slot_out = a3; return q3.z; }
   }
   *compared = n ? n : 1;
   *slot_out = NO_SLOT;
@@ -351,7 +341,7 @@ __device__ __forceinline__ u32 find_slot(const Store& st, u64 key, u32* visited,
 }
 __device__ __forceinline__ u32 find_slot_warp(const Store& st, bool active, u64 key, u32* visited, u32* id_out) {
   ProbeWindow w;
-  if (active) probe_issue(st, key, w);
+  probe_issue(st, active ? key : 0, w);          // lanes without a key read the first slots of the table and ignore them
   u32 slot;
   *id_out = probe_finish_warp(st, active, key, w, visited, &slot);
   return slot;

@@ -75,8 +75,9 @@ __device__ __forceinline__ u32 claim_slot(const Store& st, bool active, u64 key,
 #pragma unroll
     for (int x = 0; x < PROBE_WINDOW; ++x) {
       idx[x] = wrap_slot(s + x, st.slots);
-      k[x] = i == 0 ? (((u64)w.v[x].y << 32) | w.v[x].x) : *reinterpret_cast<volatile u64*>(&st.table[idx[x]].key);
+      k[x] = *reinterpret_cast<volatile u64*>(&st.table[idx[x]].key);
     }
+    if (i == 0) { k[0] = slot_key(w.v0); k[1] = slot_key(w.v1); k[2] = slot_key(w.v2); k[3] = slot_key(w.v3); }   // read already
 #pragma unroll
     for (int x = 0; x < PROBE_WINDOW; ++x) {
       if (got != NO_SLOT) break;
