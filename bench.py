@@ -43,7 +43,7 @@ NCU_READ_FACTOR = 1.00    # dram__bytes_read.sum / (distinct source blocks x blo
 NCU_WRITE_FACTOR = 0.99   # dram__bytes_write.sum / (delivered blocks x block bytes)
 FALLBACK_HBM_GBS = 6650.0
 # L2 read sectors per issued probe of lookup_kernel on the 10^6-node stress, from the ncu capture in profiles/
-L2_SECTORS_PER_PROBE = 9.3
+L2_SECTORS_PER_PROBE = 8.3
 
 
 def measured_peak():
