@@ -455,6 +455,32 @@ def test_table_under_delete_heavy_churn(table_slots):
     p.close()
 
 
+def test_table_almost_full_keys_far_from_home():
+    """1,024 blocks in a table of 1,100 slots, filled to the brim and then churned: runs of occupied slots grow to hundreds
+    of slots, so keys land beyond the exact bits and the group bits of their home slot (distance 248 and more: the far
+    bit, every slot up to the largest distance ever used is compared).  Every lookup result is compared with the oracle."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    p = Pair(sh, 1024, max_requests=8, max_batch_blocks=8 * 8, table_slots=1100)
+    rng = np.random.default_rng(12)
+    history = []
+    for step in range(15):                                   # 15 x 64 new nodes
+        batch = [rng.integers(0, 1 << 30, size=8, dtype=np.int32) for _ in range(8)]
+        p.insert(batch, 8)
+        history.append(batch)
+    for step in range(150):
+        batch = [rng.integers(0, 1 << 30, size=8, dtype=np.int32) for _ in range(8)]
+        p.evict(0, 30 + step % 40, literal=False)            # room for about half of the 64 new nodes: the rest is denied
+        p.insert(batch, 8)
+        history.append(batch)
+        p.lookup(batch, 8)
+        p.lookup(history[int(rng.integers(0, len(history)))], 8)          # an old batch: partly or wholly evicted
+        assert p.check_status() in (0, G.S_NOSPACE)
+    s = p.check_counts()
+    assert s.far_keys > 100 and s.max_displacement >= 248
+    p.close()
+
+
 @pytest.mark.parametrize("name,mk", [ENGINES[0], ENGINES[3], ENGINES[4]], ids=["vector", "bulk", "bulk_8x8k_3cta"])
 def test_many_requests_share_one_prefix(name, mk):
     """40 identical prompts: every pool block has 40 destinations (more than the per-unit destination cache holds),
