@@ -637,6 +637,33 @@ def test_maximum_depth_request():
     p.close()
 
 
+def test_maximum_depth_requests_are_looked_up_and_gathered_in_one_launch():
+    """Two requests of 65,535 and 40,000 one-token blocks over the same stored prompt: the one-launch lookup + gather with
+    block depths up to the 16 bits an owned-list entry has, every block of the shorter request shared with the longer one."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    rng = np.random.default_rng(13)
+    seq = rng.integers(0, 50000, size=65535, dtype=np.int32)
+    p = Pair(sh, 66000, max_requests=2, max_batch_blocks=2 * 65535)
+    tab = np.arange(65535, dtype=np.int32)[None, :]
+    p.insert([seq], 65535, W.random_kv_cache(5, sh, 65535), tab)
+    nd = 65535 + 40000
+    bt = np.full((2, 65535), -1, dtype=np.int32)
+    perm = rng.permutation(nd).astype(np.int32)
+    bt[0, :] = perm[:65535]
+    bt[1, :40000] = perm[65535:]
+    dst = [np.full((2, nd, sh.chunk_bytes), 0x11, dtype=np.uint8) for _ in range(sh.layers)]
+    before = p.g.launch_count()
+    s0 = p.g.stats()
+    mo, io = p.lookup_fetch([seq, seq[:40000]], 65535, dst, bt)
+    assert p.g.launch_count() - before == 1
+    assert mo.tolist() == [65535, 40000]
+    s1 = p.g.stats()
+    assert s1.blocks_fetched[0] - s0.blocks_fetched[0] == nd and s1.blocks_fetched_distinct - s0.blocks_fetched_distinct == 65535
+    assert p.check_status() == 0
+    p.close()
+
+
 @pytest.mark.parametrize("engine", ["bulk", "vector"])
 def test_chunk_sizes_that_do_not_divide_into_stages(engine):
     """Chunks of 48 KiB (a 32 KiB piece and a 16 KiB tail), 1600 B and 80 B: byte-exact insert and fetch."""
