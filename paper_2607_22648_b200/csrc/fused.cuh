@@ -207,17 +207,19 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
       const int j = (int)(w & 0xFFFFu);
       const int id = src.x;
       if (id < 0 || (u32)id >= st.n[0]) { if (q == 0) raise(st, S_BOUNDS); continue; }
-      u32 n = 0;
-      bool bad = false;
-      if (src.y < 0 || (u32)src.y >= a.pc.num_blocks) bad = true;
+      u32 n = 0, bad = 0;
+      if (src.y < 0 || (u32)src.y >= a.pc.num_blocks) ++bad;
       else s_unit_blk[n++] = (u32)src.y;
       for (u32 set = w >> 16; set; set &= set - 1) {                      // the higher requests that share the block
         const int r2 = __ffs(set) - 1;
         const int cb = a.bt[(long long)r2 * max_blocks + j];
-        if (cb < 0 || (u32)cb >= a.pc.num_blocks) bad = true;
+        if (cb < 0 || (u32)cb >= a.pc.num_blocks) ++bad;
         else s_unit_blk[n++] = (u32)cb;
       }
-      if (bad && q == 0) raise(st, S_BOUNDS);
+      if (bad && q == 0) {                         // once per block: flag it, and take the skipped entries out of the count
+        raise(st, S_BOUNDS);
+        atomicAdd(&st.ctrl->blocks_fetched[0], 0ull - (u64)bad);
+      }
       if (n == 0) continue;
       unit_n = n;
       const u32 base_piece = q * G;

@@ -814,8 +814,9 @@ def test_small_batch_of_long_prompts_is_looked_up_and_gathered_in_one_launch(pol
             after = p.g.stats()
             stored_other = min(mb, 70) // 2
             assert after.blocks_fetched_distinct - before.blocks_fetched_distinct == min(mb, 70) + stored_other   # base's and other's blocks, once each
+            assert after.blocks_fetched[0] - before.blocks_fetched[0] == sum(min(u, 70) for u in upper[:3]) + stored_other + min(mb, 70) - 3   # entries copied
         s = p.check_counts()
-        assert s.blocks_fetched[0] == s.blocks_matched
+        assert s.blocks_fetched[0] == s.blocks_matched - 5 * len(mbs)       # all but the five bad table entries per size
         p.close()
 
 
