@@ -656,11 +656,60 @@ def latency_record(args, torch, batches=(1, 4, 16), n_docs=32, doc_tokens=4096, 
                               "step_over_copy_bound": round(step_us / bound_us, 3), "gbps": round(copy_bytes / step_us / 1e3, 1)}
         status = st.status()
         assert status == 0, "status word 0x%x after the batch-%d steps" % (status, b)
+    if bmax >= 16:
+        res["lookup_fetch_cases"] = lookup_fetch_cases(torch, st, cache, docs, rng, mb, suffix_tokens, peak, sh)
     res["config"] = {"kv_shape": "32L x 8H x 128 bf16, block 16", "prompt": "%d-token stored document + %d fresh tokens" % (doc_tokens, suffix_tokens),
                      "pool_blocks": pool, "docs": n_docs, "iters": iters, "reserve_headroom": headroom,
                      "copy_bound": "bytes of the step's fetch and insert copies (read + write) / measured copy bandwidth"}
     st.close()
     return res
+
+
+def lookup_fetch_cases(torch, st, cache, docs, rng, mb, suffix_tokens, peak, sh):
+    """ptstore_lookup_fetch alone on 16-prompt batches that are not uniform: all prompts over ONE stored document (every
+    block shared: read once, written 16 times) and one prompt that hits beside fifteen that miss.  Median of 10 calls,
+    microseconds, next to the time the bytes DRAM must move (distinct blocks read + delivered blocks written) would take at
+    the measured copy bandwidth."""
+    import ctypes as C
+    from paper_2607_22648_b200 import binding as G
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    def fresh(n):
+        return rng.integers(0, 128256, size=n, dtype=np.int32)
+
+    cases = {
+        "16_prompts_over_one_document": [np.concatenate([docs[0], fresh(suffix_tokens)]) for _ in range(16)],
+        "1_prompt_hits_15_miss": [np.concatenate([docs[1], fresh(suffix_tokens)])] + [fresh(len(docs[1]) + suffix_tokens) for _ in range(15)],
+        "16_prompts_over_16_documents": [np.concatenate([docs[i], fresh(suffix_tokens)]) for i in range(16)],
+    }
+    stream = torch.cuda.current_stream().cuda_stream
+    out = {}
+    for name, seqs in cases.items():
+        toks, offs = W.ragged(seqs)
+        t, o = dev(toks), dev(offs)
+        bt = dev(rng.permutation(16 * mb).astype(np.int32).reshape(16, mb))
+        matched = torch.empty(16, dtype=torch.int32, device="cuda")
+        ids = torch.empty((16, mb), dtype=torch.int32, device="cuda")
+        args = (st.h, t.data_ptr(), o.data_ptr(), 16, mb, 0, C.byref(cache.desc), bt.data_ptr(), matched.data_ptr(), ids.data_ptr(), stream)
+        us = []
+        s0 = None
+        for k in range(13):
+            if k == 3:
+                s0 = st.stats()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(); assert G.lib.ptstore_lookup_fetch(*args) == 0; b.record(); torch.cuda.synchronize()
+            if k >= 3:
+                us.append(a.elapsed_time(b) * 1e3)
+        s1 = st.stats()
+        delivered = (s1.blocks_fetched[0] - s0.blocks_fetched[0]) / 10
+        distinct = (s1.blocks_fetched_distinct - s0.blocks_fetched_distinct) / 10
+        need = (delivered + distinct) * sh.block_bytes
+        out[name] = {"call_us": round(float(np.median(us)), 1), "blocks_delivered": delivered, "blocks_read": distinct,
+                     "dram_bound_us": round(need / (peak * 1e9) * 1e6, 1), "call_over_bound": round(float(np.median(us)) / (need / (peak * 1e9) * 1e6), 3)}
+    assert st.status() == 0
+    return out
 
 
 def ceilings_record(torch, writes_x100=274, gib=4):
