@@ -455,6 +455,33 @@ def test_table_under_delete_heavy_churn(table_slots):
     p.close()
 
 
+@pytest.mark.parametrize("pool,slots", [(5, 8), (12, 16), (20, 30), (40, 45), (100, 108)])
+def test_tiny_tables_wrap_around(pool, slots):
+    """Tables of a few slots, nearly as many blocks as slots: every window and every flagged distance wraps around the end
+    of the table, and an insert may claim the very last empty slot.  Batches never present more new blocks than there are
+    slots left, so the table cannot overflow and every result must equal the oracle's."""
+    Pair, dev, G = _imports()
+    sh = W.KVShape(1, 1, 8, 1)
+    room = slots - pool
+    p = Pair(sh, pool, max_requests=4, max_batch_blocks=4 * room, table_slots=slots)
+    rng = np.random.default_rng(pool)
+    seqs = []
+    for step in range(200):
+        batch, left = [], room
+        while left > 0 and len(batch) < 4:
+            n = int(rng.integers(1, left + 1))
+            base = seqs[int(rng.integers(0, len(seqs)))] if seqs and rng.random() < 0.5 else np.zeros(0, dtype=np.int32)
+            s = np.concatenate([base[: int(rng.integers(0, len(base) + 1))], rng.integers(0, 9, size=n, dtype=np.int32)])[:n]
+            batch.append(s); seqs.append(s); left -= n
+        p.evict(0, int(rng.integers(0, room + 2)), literal=bool(step % 2))
+        p.insert(batch, room)
+        p.lookup((batch + [seqs[int(rng.integers(0, len(seqs)))]])[:4], room)
+        assert p.check_status() in (0, G.S_NOSPACE)
+        seqs = seqs[-30:]
+    p.check_counts()
+    p.close()
+
+
 def test_table_almost_full_keys_far_from_home():
     """1,024 blocks in a table of 1,100 slots, filled to the brim and then churned: runs of occupied slots grow to hundreds
     of slots, so keys land beyond the exact bits and the group bits of their home slot (distance 248 and more: the far
