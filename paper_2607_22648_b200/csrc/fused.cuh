@@ -146,12 +146,14 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
     }
     __syncthreads();
     if (threadIdx.x < 32) {
+      if (R == 1 && lane == 0) a.taken[0] = 0;       // a single request owns all it matches: the copiers follow the lookup itself
       const int m = chain_probe_request(st, crow, nblk, r, max_blocks, a.flags, a.epoch, a.matched, a.ids_out, a.hashed, a.progress, tag, lane);
       if (lane == 0) {
         s_m = m;
         if (m) atomicAdd(&st.ctrl->blocks_fetched[0], (u64)m);
+        if (m && R == 1) atomicAdd(&st.ctrl->blocks_fetched_distinct, (u64)m);
       }
-    } else if (threadIdx.x < 64) {
+    } else if (threadIdx.x < 64 && R > 1) {
       build_owned_list(st, a, (int)r, tag, lane);
     }
     __syncthreads();
@@ -177,7 +179,7 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
   bool ok = true;
   auto await_owned = [&](int r, int need) -> bool {          // false when the wait ran out
     int count; bool fin;
-    const bool got = await_progress(a.owned_progress + r, tag, need, count, fin);
+    const bool got = await_progress((R == 1 ? a.progress : a.owned_progress) + r, tag, need, count, fin);
     s_known[r] = count; s_final[r] = fin ? 1 : 0;
     if (!got) { ok = false; raise(st, S_TIMEOUT); }
     return got;
@@ -202,8 +204,15 @@ __global__ void __launch_bounds__(LONG_THREADS) lookup_gather_kernel(Store st, F
       const u32 q = u - (u32)k * U;
       if (k >= s_known[r] && !s_final[r] && !await_owned(r, k + 1)) return false;
       if (k >= s_known[r]) { alive &= ~(1u << r); continue; }            // final and shorter: nothing left of r
-      const u32 w = __ldcg(a.owned + (long long)r * max_blocks + k);     // lists are written during this launch: not
-      const int2 src = __ldcg(a.owned_src + (long long)r * max_blocks + k);   // through L1
+      u32 w;
+      int2 src;
+      if (R == 1) {                                                       // the k-th matched block, owned, unshared
+        w = (u32)k;
+        src = make_int2(__ldcg(a.ids_out + k), a.bt[k]);
+      } else {
+        w = __ldcg(a.owned + (long long)r * max_blocks + k);              // lists are written during this launch: not
+        src = __ldcg(a.owned_src + (long long)r * max_blocks + k);        // through L1
+      }
       const int j = (int)(w & 0xFFFFu);
       const int id = src.x;
       if (id < 0 || (u32)id >= st.n[0]) { if (q == 0) raise(st, S_BOUNDS); continue; }
