@@ -18,18 +18,23 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 _lib = None
 
 
-def build_oracle(force=False):
+_SANITIZE = os.environ.get("PTSTORE_ORACLE_SANITIZE") == "1"   # checker build: AddressSanitizer + UBSan (the process must preload libasan)
+
+
+def build_oracle(force=False, sanitize=_SANITIZE):
     """Compile the oracle with g++ unless the shared object was already built from exactly this source."""
     import hashlib
-    want = hashlib.sha256(open(_SRC, "rb").read()).hexdigest()
-    stamp = _LIB + ".srchash"
-    if force or not os.path.exists(_LIB) or not os.path.exists(stamp) or open(stamp).read().strip() != want:
-        tmp = _LIB + ".tmp%d" % os.getpid()
-        subprocess.check_call(["g++", "-std=c++17", "-O2", "-Wall", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC])
-        os.replace(tmp, _LIB)
+    lib = _LIB.replace(".so", "_san.so") if sanitize else _LIB
+    flags = ["-O1", "-g", "-fno-omit-frame-pointer", "-fsanitize=address,undefined", "-fno-sanitize-recover=undefined"] if sanitize else ["-O2"]
+    want = hashlib.sha256(open(_SRC, "rb").read() + " ".join(flags).encode()).hexdigest()
+    stamp = lib + ".srchash"
+    if force or not os.path.exists(lib) or not os.path.exists(stamp) or open(stamp).read().strip() != want:
+        tmp = lib + ".tmp%d" % os.getpid()
+        subprocess.check_call(["g++", "-std=c++17"] + flags + ["-Wall", "-shared", "-fPIC", "-pthread", "-o", tmp, _SRC])
+        os.replace(tmp, lib)
         with open(stamp, "w") as f:
             f.write(want)
-    return _LIB
+    return lib
 
 
 def _load():
