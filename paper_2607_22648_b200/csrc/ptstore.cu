@@ -174,7 +174,12 @@ int launch_coop(ptstore* h, Kernel kernel, int grid, int threads, Args& args, cu
   void* params[2] = {&h->st, &args};
   cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), params, smem, s);
   h->launches += 1;
-  if (e != cudaSuccess) { (void)cudaGetLastError(); h->last_cuda = (int)e; return PTSTORE_E_CUDA; }
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    h->last_cuda = (int)e;
+    if (barrier) --h->coop_seq; else --h->gather_seq;      // the number was not used: the kernel that clears a later counter never ran
+    return PTSTORE_E_CUDA;
+  }
   return PTSTORE_OK;
 }
 
